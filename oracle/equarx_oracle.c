@@ -1,0 +1,375 @@
+/*
+ * EQuARX CPU oracle -- TEST INFRASTRUCTURE, NOT PART OF THE PRODUCT.
+ *
+ * A plain, slow, single-threaded restatement of the arithmetic that EQuARX
+ * (arXiv 2506.17615) runs beside the steps of a ring AllReduce: dynamic
+ * block-wise int8 quantization (Section 3.2), the dequantize -> fp32 add ->
+ * requantize of every reduce-scatter hop (Section 3.1), and the extra
+ * quantize/dequantize pair of the quantized all-gather (Section 3.4), in the
+ * fixed order of the full-loop ring (Section 3, Fig. 1; Section 3.3, Fig. 4).
+ *
+ * Only the tests, the smoke check and the bench's cpu_baseline / reference
+ * legs may call this file.  It shares no code, header, table or constant
+ * with the CUDA library; the CUDA library never calls it.
+ *
+ * The method is an approximation with a fixed evaluation order, so this file
+ * takes the algorithm step by step in the paper's order (ring step 0 sends a
+ * quantized shard; every later step dequantizes the received shard to fp32,
+ * adds the local counterpart, requantizes and forwards; the all-gather
+ * forwards the last message and everybody dequantizes it).  There is no
+ * blocking, fusion or reordering beyond that.  Precision is the paper's:
+ * bf16 tensors, int8 payload, fp32 accumulation ("higher precision (e.g.
+ * FP32)", Section 3.1).  Where the paper is silent the reading taken is
+ * stated next to the code:
+ *   - ring direction: rank r sends to rank (r+1) mod N; shard k ends on
+ *     rank k (the semi-loop example of Section 3.3 finishes shard 0 on
+ *     device 0).
+ *   - a block is B contiguous elements of a shard with one fp32 scale
+ *     (Fig. 3 caption: one scale per block of entries; the 8x128 strided
+ *     layout of Section 3.2 is a TPU register artefact and is not used).
+ *   - symmetric quantization to [-127, 127]: scale = amax / 127 (the
+ *     dequantization multiplier, which is what travels as metadata),
+ *     code = clamp(rne(v * (127 / amax))), both divisions IEEE fp32.
+ *   - blocks with amax < 2^-118 (zero blocks included) get scale 0 and all
+ *     codes 0, so that the scale is never subnormal and nothing depends on
+ *     flush-to-zero behaviour.
+ *   - dequantize-and-add is one fused multiply-add fmaf(code, scale, local).
+ *   - the partial sum stays fp32 between the add and the requantization.
+ *   - every rank, the owner included, outputs bf16_rne(code * scale) of the
+ *     all-gather message, so all N outputs are bit-identical.
+ *   - Inf/NaN inputs are outside the contract (status 9).
+ *
+ * Pins (tests/test_oracle_*.py): hand-worked blocks, tie and range blocks,
+ * exact-integer reductions that must equal a plain integer sum, an exact
+ * rational re-evaluation on tiny inputs, scaling / negation / permutation /
+ * rotation invariants, the a-posteriori error bound against the fp64 sum,
+ * and the mean squared errors printed in Section 4.1 (Fig. 7).
+ * Unpinned (declared choices, nothing in the paper or mathematics fixes
+ * them): the ring direction and the 2^-118 flush threshold.
+ *
+ * Build: gcc -O2 -std=c11 -ffp-contract=off -fPIC -shared (no -ffast-math).
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+enum {
+    ORACLE_OK = 0,
+    ORACLE_ERR_NULL = 1,
+    ORACLE_ERR_NRANKS = 2,
+    ORACLE_ERR_BLOCK = 3,
+    ORACLE_ERR_COUNT = 4,
+    ORACLE_ERR_ALLOC = 6,
+    ORACLE_ERR_NONFINITE = 9
+};
+
+/* bf16 <-> fp32.  bf16 is the upper half of an fp32 word, so widening is exact. */
+static float bf16_to_f32(uint16_t h)
+{
+    uint32_t u = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return f;
+}
+
+/* fp32 -> bf16, round to nearest, ties to even (finite input). */
+static uint16_t f32_to_bf16_rne(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    uint32_t keep_lsb = (u >> 16) & 1u;
+    u += 0x7FFFu + keep_lsb;
+    return (uint16_t)(u >> 16);
+}
+
+static int bf16_is_finite(uint16_t h) { return (h & 0x7F80u) != 0x7F80u; }
+
+/*
+ * Q_p1 + Q_p2 of Section 3.1 on one block of `block` fp32 values:
+ * first pass finds the metadata (max |v|), second pass scales the data.
+ */
+static void quantize_one_block(const float *v, int block, int8_t *code, float *scale_out)
+{
+    float amax = 0.0f;
+    for (int i = 0; i < block; ++i) {
+        float a = fabsf(v[i]);
+        if (a > amax) amax = a;
+    }
+    float scale, inv;
+    if (!(amax >= 0x1p-118f)) {
+        scale = 0.0f;
+        inv = 0.0f;
+    } else {
+        scale = amax / 127.0f;
+        inv = 127.0f / amax;
+    }
+    for (int i = 0; i < block; ++i) {
+        float t = v[i] * inv;
+        float r = rintf(t);          /* default rounding mode: ties to even */
+        if (r > 127.0f) r = 127.0f;
+        if (r < -127.0f) r = -127.0f;
+        code[i] = (int8_t)r;
+    }
+    *scale_out = scale;
+}
+
+static int check_block_count(size_t count, int block)
+{
+    if (block < 1) return ORACLE_ERR_BLOCK;
+    if (count == 0 || count % (size_t)block != 0) return ORACLE_ERR_COUNT;
+    return ORACLE_OK;
+}
+
+/* Ring step 0: quantize a bf16 buffer block by block (Section 3.1, 3.2). */
+int equarx_oracle_quantize_blocks(const uint16_t *x, size_t count, int block,
+                                  int8_t *codes, float *scales)
+{
+    if (!x || !codes || !scales) return ORACLE_ERR_NULL;
+    int st = check_block_count(count, block);
+    if (st) return st;
+    float *v = (float *)malloc((size_t)block * sizeof(float));
+    if (!v) return ORACLE_ERR_ALLOC;
+    for (size_t b = 0; b < count / (size_t)block; ++b) {
+        for (int i = 0; i < block; ++i) {
+            uint16_t h = x[b * (size_t)block + i];
+            if (!bf16_is_finite(h)) { free(v); return ORACLE_ERR_NONFINITE; }
+            v[i] = bf16_to_f32(h);
+        }
+        quantize_one_block(v, block, codes + b * (size_t)block, scales + b);
+    }
+    free(v);
+    return ORACLE_OK;
+}
+
+/*
+ * Ring steps 1..N-1: dequantize the received shard to fp32, add the local
+ * counterpart, requantize (Section 3.1).
+ */
+int equarx_oracle_rs_step(const int8_t *codes_in, const float *scales_in,
+                          const uint16_t *local, size_t count, int block,
+                          int8_t *codes_out, float *scales_out)
+{
+    if (!codes_in || !scales_in || !local || !codes_out || !scales_out) return ORACLE_ERR_NULL;
+    int st = check_block_count(count, block);
+    if (st) return st;
+    float *v = (float *)malloc((size_t)block * sizeof(float));
+    if (!v) return ORACLE_ERR_ALLOC;
+    for (size_t b = 0; b < count / (size_t)block; ++b) {
+        float s = scales_in[b];
+        for (int i = 0; i < block; ++i) {
+            size_t e = b * (size_t)block + i;
+            if (!bf16_is_finite(local[e])) { free(v); return ORACLE_ERR_NONFINITE; }
+            v[i] = fmaf((float)codes_in[e], s, bf16_to_f32(local[e]));
+        }
+        quantize_one_block(v, block, codes_out + b * (size_t)block, scales_out + b);
+    }
+    free(v);
+    return ORACLE_OK;
+}
+
+/* All-gather receive side: dequantize the message to bf16 (Section 3.4). */
+int equarx_oracle_ag_dequant(const int8_t *codes, const float *scales, size_t count,
+                             int block, uint16_t *out)
+{
+    if (!codes || !scales || !out) return ORACLE_ERR_NULL;
+    int st = check_block_count(count, block);
+    if (st) return st;
+    for (size_t e = 0; e < count; ++e) {
+        float d = (float)codes[e] * scales[e / (size_t)block];
+        out[e] = f32_to_bf16_rne(d);
+    }
+    return ORACLE_OK;
+}
+
+static int check_sim_args(int nranks, size_t count, int block)
+{
+    if (nranks < 1 || nranks > 4096) return ORACLE_ERR_NRANKS;
+    if (block < 1) return ORACLE_ERR_BLOCK;
+    if (count == 0 || count % ((size_t)nranks * (size_t)block) != 0) return ORACLE_ERR_COUNT;
+    return ORACLE_OK;
+}
+
+/*
+ * Full-loop ring reduce-scatter + all-gather, both stages quantized.
+ *
+ * in[r], out[r]   : nranks host pointers to `count` bf16 words each.
+ * trace_scales    : optional, float [nranks shards][nranks events][count/(nranks*block)]
+ * trace_codes     : optional, int8  [nranks shards][nranks events][count/nranks]
+ *                   event j of shard k is the message sent at ring step j by
+ *                   rank (k+1+j) mod N; event N-1 is the all-gather message.
+ * exact_sum       : optional, double[count], sum over ranks of the inputs.
+ *
+ * The loop below is the ring as the paper draws it: at every step every
+ * rank produces one message for its neighbour.  Rank r sends shard
+ * (r-1-s) mod N at step s.
+ */
+int equarx_oracle_allreduce(const uint16_t *const *in, uint16_t *const *out,
+                            int nranks, size_t count, int block,
+                            float *trace_scales, int8_t *trace_codes, double *exact_sum)
+{
+    if (!in || !out) return ORACLE_ERR_NULL;
+    int st = check_sim_args(nranks, count, block);
+    if (st) return st;
+    const size_t N = (size_t)nranks;
+    const size_t shard = count / N;
+    const size_t bps = shard / (size_t)block;   /* blocks per shard */
+    for (size_t r = 0; r < N; ++r) {
+        if (!in[r] || !out[r]) return ORACLE_ERR_NULL;
+        for (size_t e = 0; e < count; ++e)
+            if (!bf16_is_finite(in[r][e])) return ORACLE_ERR_NONFINITE;
+    }
+
+    if (exact_sum) {
+        for (size_t e = 0; e < count; ++e) {
+            double s = 0.0;
+            for (size_t r = 0; r < N; ++r) s += (double)bf16_to_f32(in[r][e]);
+            exact_sum[e] = s;
+        }
+    }
+
+    /* message held by each rank: msg[cur][r] was produced by rank r in the last step */
+    int8_t *msg_codes[2];
+    float *msg_scales[2];
+    float *v = (float *)malloc((size_t)block * sizeof(float));
+    for (int p = 0; p < 2; ++p) {
+        msg_codes[p] = (int8_t *)malloc(N * shard);
+        msg_scales[p] = (float *)malloc(N * bps * sizeof(float));
+    }
+    if (!v || !msg_codes[0] || !msg_codes[1] || !msg_scales[0] || !msg_scales[1]) {
+        free(v);
+        for (int p = 0; p < 2; ++p) { free(msg_codes[p]); free(msg_scales[p]); }
+        return ORACLE_ERR_ALLOC;
+    }
+
+    for (size_t s = 0; s < N; ++s) {            /* ring step */
+        const int cur = (int)(s & 1), prev = cur ^ 1;
+        for (size_t r = 0; r < N; ++r) {        /* every rank acts in every step */
+            const size_t k = (r + N * 2 - 1 - s) % N;      /* shard handled by rank r now */
+            const size_t left = (r + N - 1) % N;           /* the neighbour it received from */
+            const uint16_t *mine = in[r] + k * shard;
+            int8_t *oc = msg_codes[cur] + r * shard;
+            float *os = msg_scales[cur] + r * bps;
+            for (size_t b = 0; b < bps; ++b) {
+                if (s == 0) {
+                    for (int i = 0; i < block; ++i)
+                        v[i] = bf16_to_f32(mine[b * (size_t)block + i]);
+                } else {
+                    const int8_t *ic = msg_codes[prev] + left * shard + b * (size_t)block;
+                    const float sc = msg_scales[prev][left * bps + b];
+                    for (int i = 0; i < block; ++i)
+                        v[i] = fmaf((float)ic[i], sc, bf16_to_f32(mine[b * (size_t)block + i]));
+                }
+                quantize_one_block(v, block, oc + b * (size_t)block, os + b);
+            }
+            if (trace_codes)
+                memcpy(trace_codes + (k * N + s) * shard, oc, shard);
+            if (trace_scales)
+                memcpy(trace_scales + (k * N + s) * bps, os, bps * sizeof(float));
+        }
+    }
+
+    /* all-gather: after step N-1 rank k holds the message of shard k; everybody dequantizes it */
+    const int last = (int)((N - 1) & 1);
+    for (size_t k = 0; k < N; ++k) {
+        const int8_t *c = msg_codes[last] + k * shard;
+        const float *sc = msg_scales[last] + k * bps;
+        for (size_t e = 0; e < shard; ++e) {
+            uint16_t h = f32_to_bf16_rne((float)c[e] * sc[e / (size_t)block]);
+            for (size_t r = 0; r < N; ++r) out[r][k * shard + e] = h;
+        }
+    }
+
+    free(v);
+    for (int p = 0; p < 2; ++p) { free(msg_codes[p]); free(msg_scales[p]); }
+    return ORACLE_OK;
+}
+
+/*
+ * The unquantized comparator: the same ring with bf16 messages, fp32 add and
+ * a bf16 rounding at every hop ("baseline BF16 AllReduce", Section 4).
+ * Step 0 sends the raw shard; the all-gather forwards the reduced shard.
+ */
+int equarx_oracle_allreduce_bf16(const uint16_t *const *in, uint16_t *const *out,
+                                 int nranks, size_t count)
+{
+    if (!in || !out) return ORACLE_ERR_NULL;
+    if (nranks < 1 || nranks > 4096) return ORACLE_ERR_NRANKS;
+    if (count == 0 || count % (size_t)nranks != 0) return ORACLE_ERR_COUNT;
+    const size_t N = (size_t)nranks;
+    const size_t shard = count / N;
+    for (size_t r = 0; r < N; ++r) {
+        if (!in[r] || !out[r]) return ORACLE_ERR_NULL;
+        for (size_t e = 0; e < count; ++e)
+            if (!bf16_is_finite(in[r][e])) return ORACLE_ERR_NONFINITE;
+    }
+    uint16_t *msg[2];
+    msg[0] = (uint16_t *)malloc(count * sizeof(uint16_t));
+    msg[1] = (uint16_t *)malloc(count * sizeof(uint16_t));
+    if (!msg[0] || !msg[1]) { free(msg[0]); free(msg[1]); return ORACLE_ERR_ALLOC; }
+    for (size_t s = 0; s < N; ++s) {
+        const int cur = (int)(s & 1), prev = cur ^ 1;
+        for (size_t r = 0; r < N; ++r) {
+            const size_t k = (r + N * 2 - 1 - s) % N;
+            const size_t left = (r + N - 1) % N;
+            const uint16_t *mine = in[r] + k * shard;
+            uint16_t *o = msg[cur] + r * shard;
+            for (size_t e = 0; e < shard; ++e) {
+                if (s == 0) {
+                    o[e] = mine[e];
+                } else {
+                    float sum = bf16_to_f32(msg[prev][left * shard + e]) + bf16_to_f32(mine[e]);
+                    o[e] = f32_to_bf16_rne(sum);
+                }
+            }
+        }
+    }
+    const int last = (int)((N - 1) & 1);
+    for (size_t k = 0; k < N; ++k)
+        for (size_t r = 0; r < N; ++r)
+            memcpy(out[r] + k * shard, msg[last] + k * shard, shard * sizeof(uint16_t));
+    free(msg[0]);
+    free(msg[1]);
+    return ORACLE_OK;
+}
+
+/*
+ * A-posteriori error bound of the quantized AllReduce against the exact sum,
+ * from the scales of the trace: every quantize event j of a block moves a
+ * value by at most half a quantization step scale_j (plus the fp32 rounding
+ * of the multiply, the two divisions and the following fused add, together
+ * below scale_j * 2^-14); a flushed block (scale 0) drops less than 2^-118
+ * per element; the last bf16 rounding is 2^-9 relative, written against the
+ * output as 2^-7.9; 2^-133 covers subnormal roundings.
+ *
+ *   bound[e] = sum_j c_j + 2^-7.9 * |out[e]| + 2^-133,
+ *   c_j = scale_j * (0.5 + 2^-14) if scale_j > 0 else 2^-117.
+ *
+ * trace_scales as written by equarx_oracle_allreduce; out is any rank's output.
+ */
+int equarx_oracle_error_bound(const float *trace_scales, const uint16_t *out,
+                              int nranks, size_t count, int block, double *bound)
+{
+    if (!trace_scales || !out || !bound) return ORACLE_ERR_NULL;
+    int st = check_sim_args(nranks, count, block);
+    if (st) return st;
+    const size_t N = (size_t)nranks;
+    const size_t shard = count / N;
+    const size_t bps = shard / (size_t)block;
+    const double rel_out = pow(2.0, -7.9);
+    for (size_t k = 0; k < N; ++k) {
+        for (size_t b = 0; b < bps; ++b) {
+            double acc = 0.0;
+            for (size_t j = 0; j < N; ++j) {
+                double sc = (double)trace_scales[(k * N + j) * bps + b];
+                acc += sc > 0.0 ? sc * (0.5 + 0x1p-14) : 0x1p-117;
+            }
+            for (int i = 0; i < block; ++i) {
+                size_t e = k * shard + b * (size_t)block + (size_t)i;
+                bound[e] = acc + rel_out * fabs((double)bf16_to_f32(out[e])) + 0x1p-133;
+            }
+        }
+    }
+    return ORACLE_OK;
+}

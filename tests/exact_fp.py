@@ -1,0 +1,103 @@
+"""Exact rational arithmetic with explicit IEEE roundings, for brute-force pins.
+
+Nothing here calls the oracle or the CUDA library.  Values are
+``fractions.Fraction``; ``round_to`` rounds a rational to the nearest number
+representable with ``p`` significant bits and minimum exponent ``emin``
+(ties to even), which is what one IEEE operation does to its exact result.
+"""
+from fractions import Fraction
+import struct
+
+F32 = dict(p=24, emin=-126)     # binary32
+BF16 = dict(p=8, emin=-126)     # bfloat16: same exponent range, 8 significant bits
+
+
+def rint_even(q: Fraction) -> int:
+    """Nearest integer, ties to even."""
+    fl = q.numerator // q.denominator
+    rem = q - fl
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and fl % 2 == 1):
+        return fl + 1
+    return fl
+
+
+def round_to(q: Fraction, p: int, emin: int) -> Fraction:
+    if q == 0:
+        return Fraction(0)
+    sign = -1 if q < 0 else 1
+    a = abs(q)
+    # exponent e with 2^e <= a < 2^(e+1)
+    e = a.numerator.bit_length() - a.denominator.bit_length()
+    if Fraction(2) ** e > a:
+        e -= 1
+    elif Fraction(2) ** (e + 1) <= a:
+        e += 1
+    e = max(e, emin)                       # subnormals share the spacing of emin
+    ulp = Fraction(2) ** (e - (p - 1))
+    return sign * rint_even(a / ulp) * ulp
+
+
+def f32(q):
+    return round_to(Fraction(q), **F32)
+
+
+def bf16(q):
+    return round_to(Fraction(q), **BF16)
+
+
+def frac_from_bf16_word(h: int) -> Fraction:
+    (f,) = struct.unpack("<f", struct.pack("<I", (h & 0xFFFF) << 16))
+    return Fraction(f)
+
+
+def bf16_word(q: Fraction) -> int:
+    """Raw bf16 word of a value that is exactly representable in bf16."""
+    (u,) = struct.unpack("<I", struct.pack("<f", float(q)))
+    assert u & 0xFFFF == 0, "not a bf16 value"
+    return u >> 16
+
+
+def f32_word(q: Fraction) -> int:
+    (u,) = struct.unpack("<I", struct.pack("<f", float(q)))
+    assert Fraction(struct.unpack("<f", struct.pack("<I", u))[0]) == q, "not an fp32 value"
+    return u
+
+
+def quantize_block(v):
+    """v: list of Fractions that are fp32 values -> (scale Fraction, codes list[int])."""
+    amax = max(abs(t) for t in v)
+    if amax < Fraction(2) ** -118:
+        return Fraction(0), [0] * len(v)
+    scale = f32(amax / 127)
+    inv = f32(Fraction(127) / amax)
+    codes = [max(-127, min(127, rint_even(f32(t * inv)))) for t in v]
+    return scale, codes
+
+
+def chain_allreduce(words, block):
+    """words[r][i]: bf16 words, N ranks x count.  Per-shard adder chains.
+
+    Shard k is reduced along ranks k+1, k+2, ..., k (mod N); every link
+    quantizes, the next rank dequantizes with one fused multiply-add.
+    Returns (out_words[count], events) with events[(k, b, j)] = (scale, codes).
+    """
+    n_ranks = len(words)
+    count = len(words[0])
+    shard = count // n_ranks
+    out = [0] * count
+    events = {}
+    for k in range(n_ranks):
+        for b in range(shard // block):
+            idx = [k * shard + b * block + i for i in range(block)]
+            order = [(k + 1 + j) % n_ranks for j in range(n_ranks)]
+            v = [frac_from_bf16_word(words[order[0]][i]) for i in idx]
+            for j in range(n_ranks):
+                scale, codes = quantize_block(v)
+                events[(k, b, j)] = (scale, codes)
+                if j < n_ranks - 1:
+                    nxt = order[j + 1]
+                    v = [f32(c * scale + frac_from_bf16_word(words[nxt][i]))
+                         for c, i in zip(codes, idx)]
+            for c, i in zip(codes, idx):
+                out[i] = bf16_word(bf16(f32(c * scale)))
+    return out, events
