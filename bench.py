@@ -1,0 +1,402 @@
+#!/usr/bin/env python
+"""Benchmark of the simulated quantized AllReduce (EQuARX hot path) on B200.
+
+One "step" is one pass of the whole hot path -- ring step 0 (quantize), N-1
+dequantize-add-requantize steps and the all-gather dequantize -- over one
+batch of synthetic bf16 tensors, through the C ABI (equarx_allreduce_sim).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C2] [--impl ours|reference]
+
+Prints ONE JSON line.  `value` is GB/s of bf16 input reduced (2 * count *
+nranks bytes per step) with inputs resident in device memory; `e2e` is the
+same metric with pinned host buffers and the copies inside the timed region.
+With --gpus N > 1 (under torchrun) every rank runs an independent replica
+on its own GPU (the path has no inter-GPU exchange): weak scaling, no
+collective on the data path; NCCL is used for the barrier and the max only.
+`--impl reference` times the CPU oracle on a bounded sample instead.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "q-AllReduce GB/s (bf16 in) & % of HBM roofline on 1 B200, N simulated ranks"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic of one dequantize-add-requantize launch per element of a rank's shard,
+# from the ncu capture summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum
+# divided by the elements the launch processed); None until a capture exists.
+DAR_TRAFFIC_BYTES_PER_ELEMENT = None
+
+
+def workload_by_name(name):
+    from paper_2506_17615_b200 import workloads as wl
+    table = {"C1": wl.C1, "C2": wl.C2, "C3": wl.C3, "C5": wl.C5}
+    if name not in table:
+        raise SystemExit(f"unknown workload {name}; choose from {sorted(table)}")
+    return table[name]
+
+
+def algorithmic_bytes(n_ranks, count, block):
+    """Minimum bytes the schedule moves: N bf16 reads, every hop message written and read
+    once (N messages of count*(1+4/block) bytes each way), N bf16 writes."""
+    wire = count * (1.0 + 4.0 / block)
+    return 2.0 * count * n_ranks + 2.0 * n_ranks * wire + 2.0 * count * n_ranks
+
+
+def launch_bytes(kind, n_ranks, count, block):
+    wire = count * (1.0 + 4.0 / block)
+    if kind == "quantize_blocks":
+        return 2.0 * count + wire
+    if kind == "rs_step_dequant_add_requant":
+        return 2.0 * count + 2.0 * wire
+    return wire + 2.0 * count * n_ranks          # ag_dequant
+
+
+def hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the GPU works."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_id):
+        self.samples = []
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(gpu_id), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append((time.perf_counter(), line.strip()))
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self, windows):
+        """windows: list of (t0, t1) host intervals during which the GPU was busy."""
+        def parse(line):
+            p = [s.strip() for s in line.split(",")]
+            return float(p[0]), float(p[1]), p[3:7]
+        rows = []
+        for t, line in self.samples:
+            if any(a <= t <= b for a, b in windows):
+                try:
+                    rows.append(parse(line))
+                except Exception:
+                    pass
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        reasons = sorted({names[i] for _, _, fl in rows for i, v in enumerate(fl) if v.lower().startswith("active")})
+        return {"sm_mhz": statistics.median(r[0] for r in rows), "sm_max_mhz": max(r[1] for r in rows),
+                "reasons": reasons, "samples": len(rows)}
+
+
+def run_reference(args):
+    """The CPU oracle, as it stands, on the host cores: bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2506_17615_b200 import workloads as wl
+    w = workload_by_name(args.workload)
+    unit = _lcm(w.hidden, w.nranks * w.block) if w.hidden else w.nranks * w.block   # whole token rows
+    # calibrate on the smallest sample, then size a step so that the run ends in ~2 minutes
+    x = wl.as_u16(wl.make_inputs(w, count=unit))
+    t0 = time.perf_counter()
+    oracle.allreduce(x, w.block)
+    rate = unit * w.nranks / max(time.perf_counter() - t0, 1e-6)          # element-events per second
+    budget = 120.0 / (args.steps + args.warmup)
+    mult = max(1, min(w.count // unit, int(rate * budget / (unit * w.nranks))))
+    count = unit * mult
+    x = wl.as_u16(wl.make_inputs(w, count=count))
+    for _ in range(args.warmup):
+        oracle.allreduce(x, w.block)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.allreduce(x, w.block)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = 2.0 * count * w.nranks / dt / 1e9
+    sample = f"first {count} of {w.count} elements per rank of {w.name} ({count * w.nranks} element-hops per step)"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8 codes, fp32 accumulate, bf16 in/out",
+        "data": "synthetic", "config": {"workload": w.name, "nranks": w.nranks, "count_per_rank": count,
+                                        "block": w.block, "dist": w.dist},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def _gcd(a, b):
+    while b:
+        a, b = b, a % b
+    return a
+
+
+def _lcm(a, b):
+    return a // _gcd(a, b) * b
+
+
+def cpu_baseline(w):
+    """The oracle on a bounded sample of the bench workload, on this machine's host cores."""
+    import oracle
+    from paper_2506_17615_b200 import workloads as wl
+    count = w.count
+    # ~60 M element-hops per second on one core: keep the sample near 10-30 s
+    max_events = 600_000_000
+    if count * w.nranks > max_events:
+        unit = _lcm(w.hidden, w.nranks * w.block) if w.hidden else w.nranks * w.block
+        count = max(unit, max_events // w.nranks // unit * unit)
+    x = wl.as_u16(wl.make_inputs(w, count=count))
+    oracle.allreduce(x[:, :w.nranks * w.block], w.block)      # loads the library
+    reps, t_total = 0, 0.0
+    while t_total < 10.0 and reps < 20:
+        t0 = time.perf_counter()
+        oracle.allreduce(x, w.block)
+        t_total += time.perf_counter() - t0
+        reps += 1
+    dt = t_total / reps
+    part = "the full workload" if count == w.count else f"the first {count} of {w.count} elements per rank"
+    return {"value": 2.0 * count * w.nranks / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{part} of {w.name}, {reps} passes, {dt:.3f} s per pass, single thread",
+            "host_cores": os.cpu_count()}
+
+
+def max_over_ranks(ms, world, device):
+    """Slowest rank's time: the job is as fast as its slowest replica."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(bytes_per_rank_step, ms_step, world):
+    """Whole-job GB/s: every replica reduces bytes_per_rank_step in ms_step (max over ranks)."""
+    return world * bytes_per_rank_step / (ms_step * 1e-3) / 1e9
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
+    ap.add_argument("--workload", default="C2")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import paper_2506_17615_b200 as eq
+    from paper_2506_17615_b200 import workloads as wl
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    w = workload_by_name(args.workload)
+    N, count, block = w.nranks, w.count, w.block
+    in_bytes = 2 * count * N
+    # inputs of consecutive steps differ, so no step finds its inputs in the 126 MB L2
+    sets = 1 if in_bytes > 1_000_000_000 else min(64, max(2, -(-378_000_000 // (2 * in_bytes))))
+    ins, outs = [], []
+    for s in range(sets):
+        src = wl.Workload(w.name, N, count, block, w.dist, w.hidden, seed=w.seed + s)
+        x = wl.make_inputs(src, device=dev)
+        ins.append([x[r] for r in range(N)])
+        o = torch.empty_like(x)
+        outs.append([o[r] for r in range(N)])
+    wb = eq.allreduce_sim_workspace_bytes(N, count, block, False)
+    ws = torch.empty(wb, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def step(i):
+        eq.allreduce_sim(ins[i % sets], outs[i % sets], N, count, block, ws, wb, False, stream)
+
+    props = torch.cuda.get_device_properties(dev)
+    sampler = ClockSampler(f"GPU-{props.uuid}" if hasattr(props, "uuid") else local)
+    windows = []
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    h0 = time.perf_counter()
+    ev0.record()
+    for i in range(args.steps):
+        step(i)
+    ev1.record()
+    torch.cuda.synchronize()
+    windows.append((h0, time.perf_counter()))
+    barrier()
+    ms_step = max_over_ranks(ev0.elapsed_time(ev1), world, dev) / args.steps
+    value = aggregate_value(in_bytes, ms_step, world)
+
+    # per-launch durations: the same schedule, one launch at a time between CUDA events
+    reps = max(5, min(50, args.steps))
+    names = ["quantize_blocks"] + ["rs_step_dequant_add_requant"] * (N - 1) + ["ag_dequant"]
+    evs = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in names]
+           for _ in range(reps)]
+    h0 = time.perf_counter()
+    for i in range(reps):
+        for l in range(N + 1):
+            a, b = evs[i][l]
+            a.record()
+            eq.allreduce_sim_range(ins[i % sets], outs[i % sets], N, count, block, ws, wb, False, l, l, stream)
+            b.record()
+    torch.cuda.synchronize()
+    windows.append((h0, time.perf_counter()))
+    per_kernel = {}
+    for i in range(reps):
+        for l, name in enumerate(names):
+            per_kernel.setdefault(name, []).append(evs[i][l][0].elapsed_time(evs[i][l][1]))
+    kernels = {}
+    total_ms = sum(sum(v) for v in per_kernel.values())
+    for name, v in per_kernel.items():
+        avg_ms = sum(v) / len(v)
+        kernels[name] = {"launches_per_step": names.count(name), "avg_us": avg_ms * 1e3,
+                         "share": sum(v) / total_ms,
+                         "algorithmic_gbs": launch_bytes(name, N, count, block) / (avg_ms * 1e-3) / 1e9}
+    dominant = max(kernels, key=lambda k: kernels[k]["share"])
+    peak, peak_src = hbm_peak()
+    achieved = kernels[dominant]["algorithmic_gbs"]
+    traffic = None
+    if dominant == "rs_step_dequant_add_requant" and DAR_TRAFFIC_BYTES_PER_ELEMENT is not None:
+        traffic = DAR_TRAFFIC_BYTES_PER_ELEMENT * count
+    roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
+                "algorithmic_bytes_per_launch": launch_bytes(dominant, N, count, block)}
+    whole_gbs = algorithmic_bytes(N, count, block) / (ms_step * 1e-3) / 1e9
+    roofline_step = {"algorithmic_bytes_per_step": algorithmic_bytes(N, count, block), "achieved": whole_gbs,
+                     "frac_of_measured_peak": whole_gbs / peak, "frac_of_nominal_8TBs": whole_gbs / NOMINAL_HBM_GBS}
+
+    # unquantized comparator on the same GPU, same inputs
+    wb16 = eq.allreduce_sim_bf16_workspace_bytes(N, count)
+    ws16 = torch.empty(wb16, dtype=torch.uint8, device=dev)
+    for i in range(args.warmup):
+        eq.allreduce_sim_bf16(ins[i % sets], outs[i % sets], N, count, ws16, wb16, stream)
+    torch.cuda.synchronize()
+    h0 = time.perf_counter()
+    ev0.record()
+    for i in range(args.steps):
+        eq.allreduce_sim_bf16(ins[i % sets], outs[i % sets], N, count, ws16, wb16, stream)
+    ev1.record()
+    torch.cuda.synchronize()
+    windows.append((h0, time.perf_counter()))
+    ms16 = ev0.elapsed_time(ev1) / args.steps
+    bf16_sim = {"value": in_bytes / (ms16 * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms16,
+                "algorithmic_bytes_per_step": count * (8 * N - 4),
+                "frac_of_measured_peak": count * (8 * N - 4) / (ms16 * 1e-3) / 1e9 / peak}
+    del ws16
+
+    # end to end: pinned host buffers, copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        h_in = torch.empty((N, count), dtype=torch.bfloat16).pin_memory()
+        h_in.copy_(torch.stack(ins[0]).cpu())
+        h_out = torch.empty((N, count), dtype=torch.bfloat16).pin_memory()
+        d_in = torch.empty((N, count), dtype=torch.bfloat16, device=dev)
+        d_out = torch.empty((N, count), dtype=torch.bfloat16, device=dev)
+        d_ins, d_outs = [d_in[r] for r in range(N)], [d_out[r] for r in range(N)]
+
+        def e2e_step():
+            d_in.copy_(h_in, non_blocking=True)
+            eq.allreduce_sim(d_ins, d_outs, N, count, block, ws, wb, False, stream)
+            h_out.copy_(d_out, non_blocking=True)
+
+        e_steps = max(3, min(20, args.steps))
+        for _ in range(3):
+            e2e_step()
+        barrier()
+        ev0.record()
+        for _ in range(e_steps):
+            e2e_step()
+        ev1.record()
+        torch.cuda.synchronize()
+        barrier()
+        ms_e = max_over_ranks(ev0.elapsed_time(ev1), world, dev) / e_steps
+        e2e = {"value": aggregate_value(in_bytes, ms_e, world), "unit": UNIT, "h2d_bytes_per_step": in_bytes,
+               "d2h_bytes_per_step": in_bytes, "ms_per_step": ms_e, "steps": e_steps}
+        del h_in, h_out, d_in, d_out
+
+    sampler.stop()
+    clocks = sampler.summary(windows)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int8 codes, fp32 accumulate, bf16 in/out", "data": "synthetic",
+            "config": {"workload": w.name, "nranks": N, "count_per_rank": count, "block": block, "dist": w.dist,
+                       "bytes_per_rank": 2 * count, "parallelism": f"replicas x{world}" if world > 1 else "1 GPU",
+                       "l2": f"{sets} input/output sets used in rotation ({sets * 2 * in_bytes / 1e6:.0f} MB "
+                             f"working set against a 126 MB L2); no explicit flush",
+                       "pdl": os.environ.get("EQUARX_PDL", "1") != "0"},
+            "e2e": e2e, "gpu_launches": args.steps * (N + 1), "clocks": clocks,
+            "roofline": roofline, "roofline_step": roofline_step, "kernels": kernels, "bf16_sim": bf16_sim,
+            "speedup_vs_bf16_sim": value / world / bf16_sim["value"],
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(w)
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,175 @@
+/*
+ * equarx.h -- C ABI of the B200 (sm_100a) library for the arithmetic hot path
+ * of EQuARX (arXiv 2506.17615): dynamic block-wise int8 quantization and the
+ * dequantize / fp32-accumulate / requantize work that runs beside the steps
+ * of a ring AllReduce, simulated on ONE GPU over N logical ranks whose bf16
+ * buffers all live in that GPU's memory.
+ *
+ * Conventions for every function
+ *   - extern "C"; returns an EQUARX_* status; never throws, aborts or exits.
+ *   - Arguments are validated on the host first; on a validation error
+ *     nothing is launched and no CUDA call is made.
+ *   - Work is enqueued on `stream` and the call returns without
+ *     synchronising.  Device buffers must stay valid until the stream has
+ *     reached the work.  The library allocates and frees nothing: the caller
+ *     owns every buffer, including the workspace.
+ *   - Pointer tables (`in_bf16`, `out_bf16`) are HOST arrays of DEVICE
+ *     pointers; they are copied into kernel parameters during the call and
+ *     may be freed as soon as it returns.  All other pointers are DEVICE
+ *     pointers.
+ *   - bf16 tensors are raw 16-bit words; bf16 buffers must be 32-byte
+ *     aligned (they are moved with 256-bit accesses), int8 code buffers and
+ *     workspaces 16-byte aligned, scale buffers 4-byte aligned.
+ *   - `block` is the number of contiguous elements that share one fp32
+ *     scale (Section 3.2, Fig. 3: one scale factor per block of entries);
+ *     supported values 64, 128, 256, 512.
+ *   - Inputs must be finite.  Inf/NaN are outside the contract: no trap,
+ *     result unspecified.
+ *
+ * Arithmetic (identical, bit for bit, in every entry point)
+ *   amax  = max |v| over the block                      (Section 3.2, max reduction)
+ *   scale = amax / 127, inv = 127 / amax (IEEE fp32);   both 0 if amax < 2^-118
+ *   code  = rne(v * inv) in [-127, 127]                 (symmetric int8, Section 4)
+ *   hop   : v = fma((float)code, scale, (float)local)   (Section 3.1: dequantize to
+ *           FP32, add the local counterpart), then quantize v again
+ *   final : out = bf16_rne((float)code * scale)         (Section 3.4)
+ */
+#ifndef EQUARX_H_
+#define EQUARX_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Same type as cudaStream_t (which is `struct CUstream_st *`). */
+typedef struct CUstream_st *equarx_stream_t;
+
+#define EQUARX_MAX_RANKS 64
+
+enum equarx_status {
+    EQUARX_OK = 0,
+    EQUARX_ERR_NULL = 1,       /* a required pointer (or table entry) is NULL            */
+    EQUARX_ERR_NRANKS = 2,     /* nranks < 1 or > EQUARX_MAX_RANKS                       */
+    EQUARX_ERR_BLOCK = 3,      /* block not in {64, 128, 256, 512}                       */
+    EQUARX_ERR_COUNT = 4,      /* count 0, not a multiple of block (per-step calls) or
+                                  of nranks*block (simulations), or above 2^40           */
+    EQUARX_ERR_ALIGN = 5,      /* a pointer breaks the alignment rules above             */
+    EQUARX_ERR_WORKSPACE = 6,  /* workspace_bytes smaller than *_workspace_bytes()       */
+    EQUARX_ERR_ALIAS = 7,      /* buffers overlap in a way the call does not allow       */
+    EQUARX_ERR_CUDA = 8        /* a launch failed; see equarx_last_cuda_error()          */
+};
+
+/*
+ * Ring step 0 (Section 3.1: "quantize the shard, send the quantized shard and
+ * the corresponding metadata"; two phases Q_p1 = metadata, Q_p2 = scaling,
+ * fused here into one pass over registers).
+ *   x_bf16 : count bf16 words (device, read)
+ *   codes  : count int8 (device, written)
+ *   scales : count/block fp32 (device, written); scales[b] belongs to
+ *            elements [b*block, (b+1)*block)
+ * count must be a multiple of block.
+ */
+int equarx_quantize_blocks(const void *x_bf16, size_t count, int block,
+                           int8_t *codes, float *scales, equarx_stream_t stream);
+
+/*
+ * Ring steps 1..N-1 (Section 3.1: "dequantize the received shard to higher
+ * precision (e.g. FP32), and perform the addition", then quantize the partial
+ * sum for the next hop).  The fp32 partial sum lives in registers only.
+ *   codes_in, scales_in   : the received message (device, read)
+ *   local_bf16            : this rank's counterpart shard, count bf16 (device, read)
+ *   codes_out, scales_out : the message for the next hop (device, written);
+ *                           must not overlap the received message
+ */
+int equarx_rs_step_dequant_add_requant(const int8_t *codes_in, const float *scales_in,
+                                       const void *local_bf16, size_t count, int block,
+                                       int8_t *codes_out, float *scales_out,
+                                       equarx_stream_t stream);
+
+/*
+ * Receive side of the quantized all-gather (Section 3.4: the extra
+ * quantize/dequantize pair; its quantize half is the requantization of the
+ * last reduce-scatter step).
+ *   out_bf16 : count bf16 words (device, written)
+ */
+int equarx_ag_dequant(const int8_t *codes, const float *scales, size_t count, int block,
+                      void *out_bf16, equarx_stream_t stream);
+
+/*
+ * Bytes of workspace equarx_allreduce_sim needs; 0 if the arguments are
+ * invalid.  Layout, with shard = count/nranks, bps = shard/block and
+ * slots = keep_trace ? nranks*nranks : 2*nranks:
+ *   float  scales[slots][bps]    at offset 0
+ *   int8_t codes [slots][shard]  at offset round_up(4*slots*bps, 256)
+ * Without trace the slot of rank r's message at ring step s is (s&1)*nranks+r
+ * (ping-pong).  With trace the slot of shard k's event j (the message sent at
+ * step j by rank (k+1+j) mod nranks; event nranks-1 is the all-gather
+ * message) is k*nranks+j, and every message of the run is kept.
+ */
+size_t equarx_allreduce_sim_workspace_bytes(int nranks, size_t count, int block, int keep_trace);
+
+/*
+ * The whole simulated quantized AllReduce: full-loop ring reduce-scatter
+ * (Section 3, Fig. 1; adder chain of Section 3.3, Fig. 4) followed by the
+ * quantized all-gather (Section 3.4), as nranks+1 launches on `stream`:
+ * step 0 quantizes, steps 1..nranks-1 dequantize-add-requantize, the last
+ * launch dequantizes every reduced shard into all nranks outputs.  Rank r
+ * sends to rank (r+1) mod nranks; at step s it sends shard (r-1-s) mod nranks;
+ * shard k is finished on rank k.
+ *   in_bf16[r]  : count bf16 words of rank r (device, read)
+ *   out_bf16[r] : count bf16 words (device, written); out_bf16[r] == in_bf16[r]
+ *                 is allowed (in place); any other overlap between buffers is
+ *                 rejected with EQUARX_ERR_ALIAS
+ *   workspace   : equarx_allreduce_sim_workspace_bytes() bytes (device), not
+ *                 overlapping any input or output; contents on return are the
+ *                 messages as laid out above
+ * count (per rank) must be a multiple of nranks*block.
+ */
+int equarx_allreduce_sim(const void *const *in_bf16, void *const *out_bf16,
+                         int nranks, size_t count, int block,
+                         void *workspace, size_t workspace_bytes, int keep_trace,
+                         equarx_stream_t stream);
+
+/*
+ * The same schedule, restricted to launches first_launch..last_launch
+ * (inclusive) of the nranks+1 launches: launch 0 is ring step 0 (quantize),
+ * launch s in 1..nranks-1 is ring step s (dequantize-add-requantize on every
+ * rank), launch nranks is the all-gather dequantize.  Running the ranges
+ * [0,a], [a+1,b], ... [.., nranks] in order on one stream gives exactly
+ * equarx_allreduce_sim; a profiler or a bench can bracket single steps this
+ * way.  Requires 0 <= first_launch <= last_launch <= nranks, else
+ * EQUARX_ERR_COUNT.  Other arguments as for equarx_allreduce_sim.
+ */
+int equarx_allreduce_sim_range(const void *const *in_bf16, void *const *out_bf16,
+                               int nranks, size_t count, int block,
+                               void *workspace, size_t workspace_bytes, int keep_trace,
+                               int first_launch, int last_launch, equarx_stream_t stream);
+
+/* Workspace bytes of the unquantized comparator (two generations of bf16 messages: 4*count); 0 if invalid. */
+size_t equarx_allreduce_sim_bf16_workspace_bytes(int nranks, size_t count);
+
+/*
+ * Unquantized comparator (the "baseline BF16 AllReduce" of Section 4): the
+ * same ring with bf16 messages, p = bf16_rne((float)p_in + (float)local) at
+ * every hop.  Step 0 sends the raw shard, so the first hop reads its
+ * neighbour's input directly; nranks launches (nranks-1 hops + all-gather).
+ * count must be a multiple of 16*nranks.  Same aliasing rules as above.
+ */
+int equarx_allreduce_sim_bf16(const void *const *in_bf16, void *const *out_bf16,
+                              int nranks, size_t count,
+                              void *workspace, size_t workspace_bytes,
+                              equarx_stream_t stream);
+
+/* Static, human-readable name of a status. */
+const char *equarx_status_string(int status);
+
+/* The cudaError_t (as int) behind the calling thread's last EQUARX_ERR_CUDA, else 0. */
+int equarx_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EQUARX_H_ */

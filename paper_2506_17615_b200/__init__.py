@@ -1,0 +1,23 @@
+"""B200-native hot path of EQuARX (arXiv 2506.17615): block-wise int8 quantize,
+per-hop dequantize / fp32 add / requantize and all-gather dequantize of a ring
+AllReduce, simulated on one GPU over N ranks.  The work is done by
+hand-written sm_100a kernels behind a C ABI (include/equarx.h); this package
+is the thin binding.  ``workloads`` holds the seeded synthetic inputs.
+"""
+from .binding import (  # noqa: F401
+    EquarxError,
+    LIB_PATH,
+    MAX_RANKS,
+    ag_dequant,
+    allreduce_sim,
+    allreduce_sim_bf16,
+    allreduce_sim_bf16_workspace_bytes,
+    allreduce_sim_range,
+    allreduce_sim_workspace_bytes,
+    last_cuda_error,
+    lib,
+    quantize_blocks,
+    rs_step_dequant_add_requant,
+    status_string,
+    trace_views,
+)

@@ -1,0 +1,42 @@
+"""In-tree build of the CUDA library for sm_100a (nvcc cross-compiles without a GPU)."""
+import os
+import shutil
+import subprocess
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+SOURCES = [os.path.join(_HERE, "csrc", "equarx_host.cu")]
+DEPENDS = SOURCES + [os.path.join(_HERE, "csrc", "equarx_kernels.cuh"),
+                     os.path.join(os.path.dirname(_HERE), "include", "equarx.h")]
+LIB = os.path.join(_HERE, "libequarx.so")
+
+NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+              "-Xcompiler", "-fPIC", "-shared"]
+
+
+def find_nvcc():
+    for cand in (os.environ.get("NVCC"), shutil.which("nvcc"), "/usr/local/cuda/bin/nvcc"):
+        if cand and os.path.exists(cand):
+            return cand
+    return None
+
+
+def is_stale():
+    if not os.path.exists(LIB):
+        return True
+    built = os.path.getmtime(LIB)
+    return any(os.path.getmtime(p) > built for p in DEPENDS)
+
+
+def build(force=False, verbose=False):
+    """Compile libequarx.so next to this file; returns its path."""
+    if not force and not is_stale():
+        return LIB
+    nvcc = find_nvcc()
+    if nvcc is None:
+        raise RuntimeError("libequarx.so is missing or out of date and nvcc was not found; "
+                           "the CUDA library cannot be built and there is no fallback")
+    tmp = f"{LIB}.{os.getpid()}.tmp"
+    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + SOURCES
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, LIB)
+    return LIB

@@ -1,0 +1,151 @@
+"""Python binding of the C ABI in include/equarx.h (ctypes, argument marshalling only).
+
+Every function has the name of its C entry point without the ``equarx_``
+prefix, takes device pointers as integers or as objects with ``data_ptr()``
+(torch tensors), and raises :class:`EquarxError` on a non-zero status.
+There is no CPU fallback: if the library cannot be loaded the import fails.
+"""
+import ctypes
+
+from . import _build
+
+MAX_RANKS = 64
+OK, ERR_NULL, ERR_NRANKS, ERR_BLOCK, ERR_COUNT, ERR_ALIGN, ERR_WORKSPACE, ERR_ALIAS, ERR_CUDA = range(9)
+
+EXPORTS = (
+    "equarx_quantize_blocks",
+    "equarx_rs_step_dequant_add_requant",
+    "equarx_ag_dequant",
+    "equarx_allreduce_sim_workspace_bytes",
+    "equarx_allreduce_sim",
+    "equarx_allreduce_sim_range",
+    "equarx_allreduce_sim_bf16_workspace_bytes",
+    "equarx_allreduce_sim_bf16",
+    "equarx_status_string",
+    "equarx_last_cuda_error",
+)
+
+
+class EquarxError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)}")
+
+
+def _load():
+    path = _build.build()
+    lib = ctypes.CDLL(path)
+    vp, sz, ci = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int
+    lib.equarx_quantize_blocks.argtypes = [vp, sz, ci, vp, vp, vp]
+    lib.equarx_rs_step_dequant_add_requant.argtypes = [vp, vp, vp, sz, ci, vp, vp, vp]
+    lib.equarx_ag_dequant.argtypes = [vp, vp, sz, ci, vp, vp]
+    lib.equarx_allreduce_sim_workspace_bytes.argtypes = [ci, sz, ci, ci]
+    lib.equarx_allreduce_sim_workspace_bytes.restype = sz
+    lib.equarx_allreduce_sim.argtypes = [vp, vp, ci, sz, ci, vp, sz, ci, vp]
+    lib.equarx_allreduce_sim_range.argtypes = [vp, vp, ci, sz, ci, vp, sz, ci, ci, ci, vp]
+    lib.equarx_allreduce_sim_bf16_workspace_bytes.argtypes = [ci, sz]
+    lib.equarx_allreduce_sim_bf16_workspace_bytes.restype = sz
+    lib.equarx_allreduce_sim_bf16.argtypes = [vp, vp, ci, sz, vp, sz, vp]
+    lib.equarx_status_string.argtypes = [ci]
+    lib.equarx_status_string.restype = ctypes.c_char_p
+    lib.equarx_last_cuda_error.argtypes = []
+    for name in EXPORTS:
+        if getattr(lib, name).restype is None:
+            getattr(lib, name).restype = ci
+    return lib
+
+
+lib = _load()
+LIB_PATH = _build.LIB
+
+
+def _ptr(x):
+    if x is None:
+        return None
+    if hasattr(x, "data_ptr"):
+        return x.data_ptr()
+    return int(x)
+
+
+def _table(ptrs):
+    if ptrs is None:
+        return None
+    return (ctypes.c_void_p * len(ptrs))(*[_ptr(p) for p in ptrs])
+
+
+def _check(status, where):
+    if status != OK:
+        raise EquarxError(status, where)
+
+
+def status_string(status):
+    return lib.equarx_status_string(int(status)).decode()
+
+
+def last_cuda_error():
+    return lib.equarx_last_cuda_error()
+
+
+def quantize_blocks(x_bf16, count, block, codes, scales, stream=0):
+    _check(lib.equarx_quantize_blocks(_ptr(x_bf16), count, block, _ptr(codes), _ptr(scales), _ptr(stream)),
+           "equarx_quantize_blocks")
+
+
+def rs_step_dequant_add_requant(codes_in, scales_in, local_bf16, count, block, codes_out, scales_out, stream=0):
+    _check(lib.equarx_rs_step_dequant_add_requant(_ptr(codes_in), _ptr(scales_in), _ptr(local_bf16), count, block,
+                                                  _ptr(codes_out), _ptr(scales_out), _ptr(stream)),
+           "equarx_rs_step_dequant_add_requant")
+
+
+def ag_dequant(codes, scales, count, block, out_bf16, stream=0):
+    _check(lib.equarx_ag_dequant(_ptr(codes), _ptr(scales), count, block, _ptr(out_bf16), _ptr(stream)),
+           "equarx_ag_dequant")
+
+
+def allreduce_sim_workspace_bytes(nranks, count, block, keep_trace=False):
+    return lib.equarx_allreduce_sim_workspace_bytes(nranks, count, block, int(bool(keep_trace)))
+
+
+def allreduce_sim(in_bf16, out_bf16, nranks, count, block, workspace, workspace_bytes, keep_trace=False, stream=0):
+    _check(lib.equarx_allreduce_sim(_table(in_bf16), _table(out_bf16), nranks, count, block, _ptr(workspace),
+                                    workspace_bytes, int(bool(keep_trace)), _ptr(stream)),
+           "equarx_allreduce_sim")
+
+
+def allreduce_sim_range(in_bf16, out_bf16, nranks, count, block, workspace, workspace_bytes, keep_trace,
+                        first_launch, last_launch, stream=0):
+    _check(lib.equarx_allreduce_sim_range(_table(in_bf16), _table(out_bf16), nranks, count, block, _ptr(workspace),
+                                          workspace_bytes, int(bool(keep_trace)), first_launch, last_launch,
+                                          _ptr(stream)),
+           "equarx_allreduce_sim_range")
+
+
+def allreduce_sim_bf16_workspace_bytes(nranks, count):
+    return lib.equarx_allreduce_sim_bf16_workspace_bytes(nranks, count)
+
+
+def allreduce_sim_bf16(in_bf16, out_bf16, nranks, count, workspace, workspace_bytes, stream=0):
+    _check(lib.equarx_allreduce_sim_bf16(_table(in_bf16), _table(out_bf16), nranks, count, _ptr(workspace),
+                                         workspace_bytes, _ptr(stream)),
+           "equarx_allreduce_sim_bf16")
+
+
+def trace_views(workspace_u8, nranks, count, block, keep_trace=True):
+    """Split a workspace (1-D uint8 tensor or numpy array) into (scales, codes) views.
+
+    Returns (float32 [slots, bps], int8 [slots, shard]) with slots = N*N for a
+    trace ([shard k][event j] flattened) or 2*N for the ping-pong layout.
+    """
+    shard = count // nranks
+    bps = shard // block
+    slots = nranks * nranks if keep_trace else 2 * nranks
+    off = (4 * slots * bps + 255) // 256 * 256
+    if hasattr(workspace_u8, "numpy"):      # torch tensor
+        import torch
+        sc = workspace_u8[:4 * slots * bps].view(torch.float32).view(slots, bps)
+        co = workspace_u8[off:off + slots * shard].view(torch.int8).view(slots, shard)
+        return sc, co
+    import numpy as np
+    sc = workspace_u8[:4 * slots * bps].view(np.float32).reshape(slots, bps)
+    co = workspace_u8[off:off + slots * shard].view(np.int8).reshape(slots, shard)
+    return sc, co

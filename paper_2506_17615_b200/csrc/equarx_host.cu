@@ -1,0 +1,324 @@
+// C ABI of the EQuARX hot-path library: argument validation, the ring step
+// loop (full-loop reduce-scatter + quantized all-gather, Sections 3, 3.3, 3.4
+// of arXiv 2506.17615) and the launches.  Declarations and the contract of
+// every entry point are in include/equarx.h.
+#include "equarx_kernels.cuh"
+
+#include <cstdlib>
+#include <cstring>
+
+#include "../../include/equarx.h"
+
+namespace {
+
+using namespace equarx;
+
+thread_local int g_last_cuda_error = 0;
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+inline bool overlap(const void* a, size_t na, const void* b, size_t nb) {
+    const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
+    return x < y + nb && y < x + na;
+}
+
+inline int lanes_per_block(int block) {
+    switch (block) {
+        case 64: return 4;
+        case 128: return 8;
+        case 256: return 16;
+        case 512: return 32;
+        default: return 0;
+    }
+}
+
+constexpr size_t kMaxCount = size_t(1) << 40;
+
+inline int check_step_shape(size_t count, int block) {
+    if (!lanes_per_block(block)) return EQUARX_ERR_BLOCK;
+    if (count == 0 || count > kMaxCount || count % size_t(block) != 0) return EQUARX_ERR_COUNT;
+    return EQUARX_OK;
+}
+
+inline int check_sim_shape(int nranks, size_t count, int block) {
+    if (nranks < 1 || nranks > EQUARX_MAX_RANKS) return EQUARX_ERR_NRANKS;
+    if (!lanes_per_block(block)) return EQUARX_ERR_BLOCK;
+    if (count == 0 || count > kMaxCount || count % (size_t(nranks) * size_t(block)) != 0)
+        return EQUARX_ERR_COUNT;
+    return EQUARX_OK;
+}
+
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Programmatic dependent launch is on unless EQUARX_PDL=0 (read once).
+bool use_pdl() {
+    static const bool on = [] {
+        const char* e = std::getenv("EQUARX_PDL");
+        return !(e && e[0] == '0');
+    }();
+    return on;
+}
+
+template <typename Kernel, typename Args>
+int launch(Kernel kernel, dim3 grid, const Args& args, cudaStream_t stream, bool dependent) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = (dependent && use_pdl()) ? 1 : 0;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, args);
+    if (e != cudaSuccess) {
+        g_last_cuda_error = int(e);
+        (void)cudaGetLastError();
+        return EQUARX_ERR_CUDA;
+    }
+    return EQUARX_OK;
+}
+
+inline dim3 grid_for(uint64_t shard, unsigned y) {
+    const uint64_t groups = shard / kLaneElems;
+    return dim3(unsigned((groups + kThreads - 1) / kThreads), y, 1);
+}
+
+template <bool FIRST>
+int launch_step(int block, const StepArgs& a, unsigned nranks, cudaStream_t stream, bool dependent) {
+    const dim3 grid = grid_for(a.shard, nranks);
+    switch (block) {
+        case 64: return launch(rs_step_kernel<4, FIRST>, grid, a, stream, dependent);
+        case 128: return launch(rs_step_kernel<8, FIRST>, grid, a, stream, dependent);
+        case 256: return launch(rs_step_kernel<16, FIRST>, grid, a, stream, dependent);
+        default: return launch(rs_step_kernel<32, FIRST>, grid, a, stream, dependent);
+    }
+}
+
+int launch_gather(int block, const GatherArgs& a, cudaStream_t stream, bool dependent) {
+    const dim3 grid = grid_for(a.shard, a.nranks);
+    switch (block) {
+        case 64: return launch(ag_dequant_kernel<4>, grid, a, stream, dependent);
+        case 128: return launch(ag_dequant_kernel<8>, grid, a, stream, dependent);
+        case 256: return launch(ag_dequant_kernel<16>, grid, a, stream, dependent);
+        default: return launch(ag_dequant_kernel<32>, grid, a, stream, dependent);
+    }
+}
+
+// in/out tables of a simulation: NULLs, alignment, overlap.  out[r] == in[r] is the
+// one overlap allowed.
+int check_tables(const void* const* in, void* const* out, int nranks, size_t bytes,
+                 const void* ws, size_t ws_bytes) {
+    if (!in || !out) return EQUARX_ERR_NULL;
+    for (int r = 0; r < nranks; ++r)
+        if (!in[r] || !out[r]) return EQUARX_ERR_NULL;
+    for (int r = 0; r < nranks; ++r)
+        if (!aligned(in[r], 32) || !aligned(out[r], 32)) return EQUARX_ERR_ALIGN;
+    for (int r = 0; r < nranks; ++r) {
+        for (int q = 0; q < nranks; ++q) {
+            if (q != r && overlap(out[r], bytes, out[q], bytes)) return EQUARX_ERR_ALIAS;
+            if (overlap(out[r], bytes, in[q], bytes) && !(q == r && out[r] == in[r]))
+                return EQUARX_ERR_ALIAS;
+        }
+        if (ws && (overlap(ws, ws_bytes, in[r], bytes) || overlap(ws, ws_bytes, out[r], bytes)))
+            return EQUARX_ERR_ALIAS;
+    }
+    return EQUARX_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* equarx_status_string(int status) {
+    switch (status) {
+        case EQUARX_OK: return "EQUARX_OK";
+        case EQUARX_ERR_NULL: return "EQUARX_ERR_NULL: a required pointer is NULL";
+        case EQUARX_ERR_NRANKS: return "EQUARX_ERR_NRANKS: nranks outside [1, 64]";
+        case EQUARX_ERR_BLOCK: return "EQUARX_ERR_BLOCK: block must be 64, 128, 256 or 512";
+        case EQUARX_ERR_COUNT: return "EQUARX_ERR_COUNT: count is 0, too large or not a multiple of the required unit";
+        case EQUARX_ERR_ALIGN: return "EQUARX_ERR_ALIGN: a pointer is not aligned as required";
+        case EQUARX_ERR_WORKSPACE: return "EQUARX_ERR_WORKSPACE: workspace too small";
+        case EQUARX_ERR_ALIAS: return "EQUARX_ERR_ALIAS: buffers overlap";
+        case EQUARX_ERR_CUDA: return "EQUARX_ERR_CUDA: a kernel launch failed";
+        default: return "EQUARX: unknown status";
+    }
+}
+
+int equarx_last_cuda_error(void) { return g_last_cuda_error; }
+
+int equarx_quantize_blocks(const void* x_bf16, size_t count, int block, int8_t* codes, float* scales,
+                           equarx_stream_t stream) {
+    if (!x_bf16 || !codes || !scales) return EQUARX_ERR_NULL;
+    if (int st = check_step_shape(count, block)) return st;
+    if (!aligned(x_bf16, 32) || !aligned(codes, 16) || !aligned(scales, 4)) return EQUARX_ERR_ALIGN;
+    if (overlap(x_bf16, 2 * count, codes, count) || overlap(x_bf16, 2 * count, scales, 4 * (count / block)) ||
+        overlap(codes, count, scales, 4 * (count / block)))
+        return EQUARX_ERR_ALIAS;
+    StepArgs a = {};
+    a.x[0] = x_bf16;
+    a.codes_out = codes;
+    a.scales_out = scales;
+    a.shard = count;
+    a.bps = count / size_t(block);
+    return launch_step<true>(block, a, 1, stream, false);
+}
+
+int equarx_rs_step_dequant_add_requant(const int8_t* codes_in, const float* scales_in, const void* local_bf16,
+                                       size_t count, int block, int8_t* codes_out, float* scales_out,
+                                       equarx_stream_t stream) {
+    if (!codes_in || !scales_in || !local_bf16 || !codes_out || !scales_out) return EQUARX_ERR_NULL;
+    if (int st = check_step_shape(count, block)) return st;
+    if (!aligned(local_bf16, 32) || !aligned(codes_in, 16) || !aligned(codes_out, 16) || !aligned(scales_in, 4) ||
+        !aligned(scales_out, 4))
+        return EQUARX_ERR_ALIGN;
+    const size_t sb = 4 * (count / size_t(block));
+    const void* bufs[5] = {codes_in, scales_in, local_bf16, codes_out, scales_out};
+    const size_t lens[5] = {count, sb, 2 * count, count, sb};
+    for (int i = 0; i < 5; ++i)
+        for (int j = 3; j < 5; ++j)
+            if (i != j && overlap(bufs[i], lens[i], bufs[j], lens[j])) return EQUARX_ERR_ALIAS;
+    StepArgs a = {};
+    a.x[0] = local_bf16;
+    a.codes_in = codes_in;
+    a.scales_in = scales_in;
+    a.codes_out = codes_out;
+    a.scales_out = scales_out;
+    a.shard = count;
+    a.bps = count / size_t(block);
+    return launch_step<false>(block, a, 1, stream, false);
+}
+
+int equarx_ag_dequant(const int8_t* codes, const float* scales, size_t count, int block, void* out_bf16,
+                      equarx_stream_t stream) {
+    if (!codes || !scales || !out_bf16) return EQUARX_ERR_NULL;
+    if (int st = check_step_shape(count, block)) return st;
+    if (!aligned(out_bf16, 32) || !aligned(codes, 16) || !aligned(scales, 4)) return EQUARX_ERR_ALIGN;
+    if (overlap(out_bf16, 2 * count, codes, count) || overlap(out_bf16, 2 * count, scales, 4 * (count / block)))
+        return EQUARX_ERR_ALIAS;
+    GatherArgs a = {};
+    a.out[0] = out_bf16;
+    a.codes = codes;
+    a.scales = scales;
+    a.shard = count;
+    a.bps = count / size_t(block);
+    a.nranks = 1;
+    return launch_gather(block, a, stream, false);
+}
+
+size_t equarx_allreduce_sim_workspace_bytes(int nranks, size_t count, int block, int keep_trace) {
+    if (check_sim_shape(nranks, count, block) != EQUARX_OK) return 0;
+    const size_t N = size_t(nranks), shard = count / N, bps = shard / size_t(block);
+    const size_t slots = keep_trace ? N * N : 2 * N;
+    return round_up(4 * slots * bps, 256) + slots * shard;
+}
+
+int equarx_allreduce_sim(const void* const* in_bf16, void* const* out_bf16, int nranks, size_t count, int block,
+                         void* workspace, size_t workspace_bytes, int keep_trace, equarx_stream_t stream) {
+    return equarx_allreduce_sim_range(in_bf16, out_bf16, nranks, count, block, workspace, workspace_bytes,
+                                      keep_trace, 0, nranks, stream);
+}
+
+int equarx_allreduce_sim_range(const void* const* in_bf16, void* const* out_bf16, int nranks, size_t count,
+                               int block, void* workspace, size_t workspace_bytes, int keep_trace,
+                               int first_launch, int last_launch, equarx_stream_t stream) {
+    if (int st = check_sim_shape(nranks, count, block)) return st;
+    if (first_launch < 0 || first_launch > last_launch || last_launch > nranks) return EQUARX_ERR_COUNT;
+    if (!workspace) return EQUARX_ERR_NULL;
+    const size_t need = equarx_allreduce_sim_workspace_bytes(nranks, count, block, keep_trace);
+    if (workspace_bytes < need) return EQUARX_ERR_WORKSPACE;
+    if (!aligned(workspace, 16)) return EQUARX_ERR_ALIGN;
+    if (int st = check_tables(in_bf16, out_bf16, nranks, 2 * count, workspace, need)) return st;
+
+    const uint32_t N = uint32_t(nranks);
+    const size_t shard = count / N, bps = shard / size_t(block);
+    const size_t slots = keep_trace ? size_t(N) * N : 2 * size_t(N);
+    float* scales = static_cast<float*>(workspace);
+    int8_t* codes = static_cast<int8_t*>(workspace) + round_up(4 * slots * bps, 256);
+
+    // shard that rank r sends at step s, and where that message is kept
+    auto shard_of = [N](uint32_t s, uint32_t r) { return (r + 2 * N - 1 - s % N) % N; };
+    auto slot_of = [&](uint32_t s, uint32_t r) {
+        return keep_trace ? shard_of(s, r) * N + s : (s & 1u) * N + r;
+    };
+
+    StepArgs a = {};
+    a.codes_in = codes;
+    a.scales_in = scales;
+    a.codes_out = codes;
+    a.scales_out = scales;
+    a.shard = shard;
+    a.bps = bps;
+    const uint32_t first = uint32_t(first_launch), last = uint32_t(last_launch);
+    for (uint32_t s = first; s < N && s <= last; ++s) {
+        for (uint32_t r = 0; r < N; ++r) {
+            a.x[r] = static_cast<const char*>(in_bf16[r]) + size_t(shard_of(s, r)) * shard * 2;
+            a.out_slot[r] = slot_of(s, r);
+            a.in_slot[r] = s ? slot_of(s - 1, (r + N - 1) % N) : 0;
+        }
+        // only a launch that follows another launch of this call may overlap its predecessor
+        const int st = s == 0 ? launch_step<true>(block, a, N, stream, false)
+                              : launch_step<false>(block, a, N, stream, s > first);
+        if (st) return st;
+    }
+    if (last < N) return EQUARX_OK;
+
+    GatherArgs g = {};
+    for (uint32_t k = 0; k < N; ++k) {
+        g.out[k] = out_bf16[k];
+        g.slot[k] = slot_of(N - 1, k);     // after step N-1 rank k holds shard k
+    }
+    g.codes = codes;
+    g.scales = scales;
+    g.shard = shard;
+    g.bps = bps;
+    g.nranks = N;
+    return launch_gather(block, g, stream, first < N);
+}
+
+size_t equarx_allreduce_sim_bf16_workspace_bytes(int nranks, size_t count) {
+    if (nranks < 1 || nranks > EQUARX_MAX_RANKS) return 0;
+    if (count == 0 || count > kMaxCount || count % (size_t(nranks) * kLaneElems) != 0) return 0;
+    return 4 * count;
+}
+
+int equarx_allreduce_sim_bf16(const void* const* in_bf16, void* const* out_bf16, int nranks, size_t count,
+                              void* workspace, size_t workspace_bytes, equarx_stream_t stream) {
+    if (nranks < 1 || nranks > EQUARX_MAX_RANKS) return EQUARX_ERR_NRANKS;
+    if (count == 0 || count > kMaxCount || count % (size_t(nranks) * kLaneElems) != 0) return EQUARX_ERR_COUNT;
+    if (!workspace) return EQUARX_ERR_NULL;
+    const size_t need = 4 * count;
+    if (workspace_bytes < need) return EQUARX_ERR_WORKSPACE;
+    if (!aligned(workspace, 32)) return EQUARX_ERR_ALIGN;
+    if (int st = check_tables(in_bf16, out_bf16, nranks, 2 * count, workspace, need)) return st;
+
+    const uint32_t N = uint32_t(nranks);
+    const size_t shard = count / N;
+    char* ws = static_cast<char*>(workspace);
+    auto shard_of = [N](uint32_t s, uint32_t r) { return (r + 2 * N - 1 - s % N) % N; };
+    auto msg = [&](uint32_t s, uint32_t r) { return ws + (size_t(s & 1u) * N + r) * shard * 2; };
+
+    Bf16StepArgs a = {};
+    a.shard = shard;
+    for (uint32_t s = 1; s < N; ++s) {
+        for (uint32_t r = 0; r < N; ++r) {
+            const uint32_t left = (r + N - 1) % N, k = shard_of(s, r);
+            a.local[r] = static_cast<const char*>(in_bf16[r]) + size_t(k) * shard * 2;
+            // step 0 sends the raw shard: the first hop reads the neighbour's input in place
+            a.recv[r] = s == 1 ? static_cast<const char*>(in_bf16[left]) + size_t(k) * shard * 2 : msg(s - 1, left);
+            a.send[r] = msg(s, r);
+        }
+        if (int st = launch(bf16_step_kernel, grid_for(shard, N), a, stream, s > 1)) return st;
+    }
+    Bf16GatherArgs g = {};
+    g.shard = shard;
+    g.nranks = N;
+    for (uint32_t k = 0; k < N; ++k) {
+        g.out[k] = out_bf16[k];
+        g.src[k] = N == 1 ? in_bf16[0] : msg(N - 1, k);
+    }
+    return launch(bf16_gather_kernel, grid_for(shard, N), g, stream, N > 1);
+}
+
+}  // extern "C"

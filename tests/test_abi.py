@@ -1,0 +1,142 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports
+every function include/equarx.h declares, and rejects bad arguments before
+touching CUDA (fake, never dereferenced device addresses are enough)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2506_17615_b200 as eq
+from paper_2506_17615_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+A = 0x7000_0000_0000          # a made-up, well aligned "device address"
+MB = 1 << 20
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "equarx.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(equarx_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_function():
+    names = declared_functions()
+    assert len(names) >= 9
+    raw = ctypes.CDLL(eq.LIB_PATH)
+    for name in names:
+        assert hasattr(raw, name), name
+    assert sorted(binding.EXPORTS) == names
+
+
+def test_binding_has_the_same_names():
+    for name in declared_functions():
+        assert hasattr(eq, name[len("equarx_"):]), name
+
+
+def test_status_strings():
+    for st in range(9):
+        s = eq.status_string(st)
+        assert s.startswith("EQUARX_")
+    assert "unknown" in eq.status_string(99)
+
+
+def test_workspace_bytes():
+    # N=4, n=65536, B=256: shard 16384, 64 blocks per shard
+    assert eq.allreduce_sim_workspace_bytes(4, 65536, 256, False) == 8 * 64 * 4 + 8 * 16384
+    assert eq.allreduce_sim_workspace_bytes(4, 65536, 256, True) == 16 * 64 * 4 + 16 * 16384
+    # scales region is padded to 256 bytes: N=1, one block
+    assert eq.allreduce_sim_workspace_bytes(1, 64, 64, False) == 256 + 2 * 64
+    assert eq.allreduce_sim_workspace_bytes(3, 65536, 256, False) == 0      # not divisible
+    assert eq.allreduce_sim_workspace_bytes(4, 65536, 100, False) == 0
+    assert eq.allreduce_sim_workspace_bytes(65, 65 * 256, 256, False) == 0
+    assert eq.allreduce_sim_bf16_workspace_bytes(4, 65536) == 4 * 65536
+    assert eq.allreduce_sim_bf16_workspace_bytes(4, 65530) == 0
+
+
+def status_of(fn, *args, **kw):
+    try:
+        fn(*args, **kw)
+    except eq.EquarxError as e:
+        return e.status
+    return 0
+
+
+def test_per_step_calls_reject_bad_arguments():
+    q = eq.quantize_blocks
+    assert status_of(q, 0, 256, 256, A + MB, A + 2 * MB) == binding.ERR_NULL
+    assert status_of(q, A, 256, 96, A + MB, A + 2 * MB) == binding.ERR_BLOCK
+    assert status_of(q, A, 0, 256, A + MB, A + 2 * MB) == binding.ERR_COUNT
+    assert status_of(q, A, 300, 256, A + MB, A + 2 * MB) == binding.ERR_COUNT
+    assert status_of(q, A + 16, 256, 256, A + MB, A + 2 * MB) == binding.ERR_ALIGN   # bf16 needs 32 bytes
+    assert status_of(q, A, 256, 256, A + MB + 8, A + 2 * MB) == binding.ERR_ALIGN
+    assert status_of(q, A, 256, 256, A + MB, A + 2 * MB + 2) == binding.ERR_ALIGN
+    assert status_of(q, A, 256, 256, A + 256, A + 2 * MB) == binding.ERR_ALIAS       # codes inside x
+
+    s = eq.rs_step_dequant_add_requant
+    ok = dict(codes_in=A, scales_in=A + MB, local_bf16=A + 2 * MB, count=512, block=128,
+              codes_out=A + 3 * MB, scales_out=A + 4 * MB)
+    for key in ("codes_in", "scales_in", "local_bf16", "codes_out", "scales_out"):
+        assert status_of(s, **{**ok, key: 0}) == binding.ERR_NULL
+    assert status_of(s, **{**ok, "block": 32}) == binding.ERR_BLOCK
+    assert status_of(s, **{**ok, "count": 520}) == binding.ERR_COUNT
+    assert status_of(s, **{**ok, "codes_out": A}) == binding.ERR_ALIAS               # in place is not allowed
+    assert status_of(s, **{**ok, "scales_out": A + MB}) == binding.ERR_ALIAS
+    assert status_of(s, **{**ok, "local_bf16": A + 2 * MB + 16}) == binding.ERR_ALIGN
+
+    d = eq.ag_dequant
+    assert status_of(d, A, A + MB, 512, 512, 0) == binding.ERR_NULL
+    assert status_of(d, A, A + MB, 512, 1024, A + 2 * MB) == binding.ERR_BLOCK
+    assert status_of(d, A, A + MB, 512, 512, A + 2 * MB + 8) == binding.ERR_ALIGN
+    assert status_of(d, A, A + MB, 512, 512, A) == binding.ERR_ALIAS
+
+
+def sim_args(nranks=4, count=65536, block=256, in_place=False):
+    ins = [A + r * 16 * MB for r in range(nranks)]
+    outs = ins if in_place else [A + (64 + r) * 16 * MB for r in range(nranks)]
+    ws = A + 200 * 16 * MB
+    wb = eq.allreduce_sim_workspace_bytes(nranks, count, block)
+    return dict(in_bf16=ins, out_bf16=list(outs), nranks=nranks, count=count, block=block,
+                workspace=ws, workspace_bytes=wb)
+
+
+def test_sim_rejects_bad_arguments():
+    f = eq.allreduce_sim
+    a = sim_args()
+    assert status_of(f, **{**a, "nranks": 0}) == binding.ERR_NRANKS
+    assert status_of(f, **{**a, "nranks": 65}) == binding.ERR_NRANKS
+    assert status_of(f, **{**a, "block": 100}) == binding.ERR_BLOCK
+    assert status_of(f, **{**a, "count": 65536 + 256}) == binding.ERR_COUNT   # not a multiple of N*B
+    assert status_of(f, **{**a, "workspace": 0}) == binding.ERR_NULL
+    assert status_of(f, **{**a, "workspace_bytes": a["workspace_bytes"] - 1}) == binding.ERR_WORKSPACE
+    assert status_of(f, **{**a, "workspace": a["workspace"] + 8}) == binding.ERR_ALIGN
+    bad = dict(a); bad["in_bf16"] = a["in_bf16"][:3] + [0]
+    assert status_of(f, **bad) == binding.ERR_NULL
+    bad = dict(a); bad["out_bf16"] = [a["out_bf16"][0] + 16] + a["out_bf16"][1:]
+    assert status_of(f, **bad) == binding.ERR_ALIGN
+    bad = dict(a); bad["out_bf16"] = [a["in_bf16"][1]] + a["out_bf16"][1:]     # out[0] on another rank's input
+    assert status_of(f, **bad) == binding.ERR_ALIAS
+    bad = dict(a); bad["out_bf16"] = [a["in_bf16"][0] + 64] + a["out_bf16"][1:]  # partial overlap with own input
+    assert status_of(f, **bad) == binding.ERR_ALIAS
+    bad = dict(a); bad["out_bf16"] = [a["out_bf16"][1]] + a["out_bf16"][1:]     # two outputs share a buffer
+    assert status_of(f, **bad) == binding.ERR_ALIAS
+    bad = dict(a); bad["workspace"] = a["in_bf16"][2]
+    assert status_of(f, **bad) == binding.ERR_ALIAS
+    assert status_of(f, None, a["out_bf16"], 4, 65536, 256, a["workspace"], a["workspace_bytes"]) == binding.ERR_NULL
+
+
+def test_bf16_sim_rejects_bad_arguments():
+    f = eq.allreduce_sim_bf16
+    ins = [A + r * 16 * MB for r in range(4)]
+    outs = [A + (64 + r) * 16 * MB for r in range(4)]
+    ws = A + 200 * 16 * MB
+    assert status_of(f, ins, outs, 0, 65536, ws, 4 * 65536) == binding.ERR_NRANKS
+    assert status_of(f, ins, outs, 4, 65536 + 8, ws, 4 * 65536 + 32) == binding.ERR_COUNT
+    assert status_of(f, ins, outs, 4, 65536, 0, 4 * 65536) == binding.ERR_NULL
+    assert status_of(f, ins, outs, 4, 65536, ws, 4 * 65536 - 1) == binding.ERR_WORKSPACE
+    assert status_of(f, ins, [ins[1]] + outs[1:], 4, 65536, ws, 4 * 65536) == binding.ERR_ALIAS
+
+
+def test_no_cuda_error_recorded_by_validation():
+    assert eq.last_cuda_error() == 0

@@ -1,0 +1,212 @@
+"""GPU parity tests: the CUDA library, called through its C ABI, against the CPU
+oracle on the same seeded inputs.  Bar: bit-exact int8 codes, bit-exact fp32
+scales, and 0-ulp bf16 outputs (there is no op-order freedom in the path: the
+max is order independent and every rounding step is an explicit IEEE op)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2506_17615_b200 as eq
+from paper_2506_17615_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+BLOCKS = (64, 128, 256, 512)
+
+
+def _values(kind, count, seed):
+    g = torch.Generator().manual_seed(seed)
+    if kind == "normal":
+        v = torch.randn(count, generator=g)
+    elif kind == "wide":        # 40 binades per tensor: exercises scale range and tiny/huge ratios
+        v = torch.randn(count, generator=g) * torch.exp2(torch.randint(-20, 20, (count,), generator=g).float())
+    elif kind == "halves":      # exact .5 products against a block max of 127: ties
+        v = torch.randint(-254, 255, (count,), generator=g).float() / 2.0
+        v[::64] = 127.0
+    elif kind == "tiny":        # around the flush threshold and among bf16 subnormals
+        v = (torch.randint(-127, 128, (count,), generator=g).double()
+             * torch.exp2(torch.randint(-133, -112, (count,), generator=g).double()))
+    elif kind == "huge":        # close to the bf16 maximum
+        v = torch.randn(count, generator=g).double() * 2.0 ** 125
+    elif kind == "zeros":
+        v = torch.zeros(count)
+        v[1::7] = -0.0
+    else:
+        raise ValueError(kind)
+    return v.to(torch.bfloat16)
+
+
+KINDS = ("normal", "wide", "halves", "tiny", "huge", "zeros")
+
+
+@pytest.fixture(scope="module")
+def gu():
+    import gpu_util
+    return gpu_util
+
+
+@pytest.mark.parametrize("block", BLOCKS)
+@pytest.mark.parametrize("kind", KINDS)
+def test_step_kernels_match_oracle(gu, block, kind):
+    """quantize -> hop -> hop -> all-gather dequantize on one buffer; several 4096-element
+    tiles plus a ragged tail of 5 blocks."""
+    count = 3 * 4096 + 5 * block
+    x = [_values(kind, count, 100 + i) for i in range(3)]
+    xw = [wl.as_u16(t) for t in x]
+    xd = [t.cuda() for t in x]
+    nb = count // block
+    codes = [gu.Guarded(count) for _ in range(3)]
+    scales = [gu.Guarded(4 * nb) for _ in range(3)]
+    out = gu.Guarded(2 * count)
+    s = gu.stream_handle()
+    eq.quantize_blocks(xd[0], count, block, codes[0], scales[0], s)
+    eq.rs_step_dequant_add_requant(codes[0], scales[0], xd[1], count, block, codes[1], scales[1], s)
+    eq.rs_step_dequant_add_requant(codes[1], scales[1], xd[2], count, block, codes[2], scales[2], s)
+    eq.ag_dequant(codes[2], scales[2], count, block, out, s)
+    torch.cuda.synchronize()
+    for b in codes + scales + [out]:
+        b.check()
+    c0, s0 = oracle.quantize_blocks(xw[0], block)
+    c1, s1 = oracle.rs_step(c0, s0, xw[1], block)
+    c2, s2 = oracle.rs_step(c1, s1, xw[2], block)
+    o = oracle.ag_dequant(c2, s2, block)
+    for i, (c, sc) in enumerate(((c0, s0), (c1, s1), (c2, s2))):
+        assert np.array_equal(codes[i].view(torch.int8).cpu().numpy(), c), f"codes of event {i}"
+        assert np.array_equal(scales[i].view(torch.float32).cpu().numpy().view(np.uint32), sc.view(np.uint32)), \
+            f"scales of event {i}"
+    gu.assert_same_words(out.view(torch.bfloat16), o, "all-gather output")
+
+
+@pytest.mark.parametrize("block", BLOCKS)
+def test_single_block_and_one_tile_edges(gu, block):
+    for count in (block, 4096, 4096 + block):
+        if count % block:
+            continue
+        x = _values("normal", count, count)
+        c = gu.Guarded(count)
+        sc = gu.Guarded(4 * (count // block))
+        eq.quantize_blocks(x.cuda(), count, block, c, sc, gu.stream_handle())
+        torch.cuda.synchronize()
+        c.check(); sc.check()
+        ec, es = oracle.quantize_blocks(wl.as_u16(x), block)
+        assert np.array_equal(c.view(torch.int8).cpu().numpy(), ec)
+        assert np.array_equal(sc.view(torch.float32).cpu().numpy().view(np.uint32), es.view(np.uint32))
+
+
+def _compare_full(gu, x, block, in_place=False):
+    n_ranks, count = x.shape
+    xd = x.cuda()
+    out, ws = gu.run_sim(xd, block, keep_trace=True, in_place=in_place)
+    res = oracle.allreduce(wl.as_u16(x), block, trace=True)
+    sc, co = eq.trace_views(ws.u8, n_ranks, count, block, keep_trace=True)
+    assert np.array_equal(co.cpu().numpy().reshape(res["codes"].shape), res["codes"]), "trace codes"
+    assert np.array_equal(sc.cpu().numpy().view(np.uint32).reshape(res["scales"].shape),
+                          res["scales"].view(np.uint32)), "trace scales"
+    gu.assert_same_words(out, res["out"], "outputs")
+    # the ping-pong (no trace) path is what the bench runs: same outputs
+    out2, _ = gu.run_sim(xd, block, keep_trace=False, in_place=in_place)
+    assert torch.equal(out2.view(torch.int16), out.view(torch.int16))
+
+
+def test_config1_small_normal_full(gu):
+    x = wl.make_inputs(wl.C1)
+    _compare_full(gu, x, wl.C1.block)
+
+
+@pytest.mark.parametrize("nranks", (1, 2, 3, 5, 8, 16, 64))
+@pytest.mark.parametrize("block", BLOCKS)
+def test_rank_counts_and_blocks(gu, nranks, block):
+    # 5 blocks per shard for the large blocks (ragged vs the 4096-element tile), more for small ones
+    bps = 5 if block >= 256 else 37
+    w = wl.Workload("t", nranks, nranks * bps * block, block, "normal", seed=nranks)
+    _compare_full(gu, wl.make_inputs(w), block)
+
+
+@pytest.mark.parametrize("w,rows", [(wl.C2, 32), (wl.C3, 32)])
+def test_activation_shaped_configs_reduced(gu, w, rows):
+    """Configs 2 and 3 with fewer token rows (same hidden size, outlier channels, distribution)."""
+    count = rows * w.hidden
+    assert count % (w.nranks * w.block) == 0
+    _compare_full(gu, wl.make_inputs(w, count=count), w.block)
+
+
+def test_stress_config_reduced(gu):
+    w = wl.C5
+    _compare_full(gu, wl.make_inputs(w, count=64 * 256 * 16), 256)
+
+
+def test_in_place(gu):
+    w = wl.Workload("t", 8, 8 * 256 * 33, 256, "normal", seed=5)
+    _compare_full(gu, wl.make_inputs(w), 256, in_place=True)
+
+
+@pytest.mark.parametrize("w", [wl.C2, wl.C3, wl.C5], ids=lambda w: w.name)
+def test_full_size_sampled(gu, w):
+    """Full-size configs in the launch configuration the bench times (ping-pong workspace):
+    outputs of sampled blocks bit for bit, plus properties that hold at any size."""
+    x = wl.make_inputs(w, device="cuda")
+    out, ws = gu.run_sim(x, w.block, keep_trace=False)
+    for r in range(1, w.nranks):
+        assert torch.equal(out[0].view(torch.int16), out[r].view(torch.int16)), "outputs differ across ranks"
+    bps = w.count // w.nranks // w.block
+    picks = gu.sample_blocks(w.nranks, bps, 24, seed=1)
+    exp = gu.oracle_out_on_samples(x, picks, w.block)
+    got = gu.gather_blocks(out, picks, w.block)
+    gu.assert_same_words(got, exp, "sampled outputs")
+    # the last two messages of every rank are still in the workspace: codes within +-127
+    # and, per block, scale 0 or at least one |code| == 127
+    sc, co = eq.trace_views(ws.u8, w.nranks, w.count, w.block, keep_trace=False)
+    assert int(co.min()) >= -127
+    amax = co.view(2 * w.nranks, -1, w.block).abs().amax(dim=2)
+    assert bool(((amax == 127) | (sc == 0)).all())
+    assert bool(((sc != 0) | (amax == 0)).all())
+
+
+@pytest.mark.parametrize("nranks,count", [(1, 4096), (2, 2 * 4096 + 32), (4, 65536), (7, 7 * 16 * 301), (64, 64 * 4096)])
+def test_bf16_comparator_matches_oracle(gu, nranks, count):
+    w = wl.Workload("t", nranks, count, 256, "normal", seed=3)
+    x = wl.make_inputs(w)
+    xd = x.cuda()
+    wb = eq.allreduce_sim_bf16_workspace_bytes(nranks, count)
+    ws = gu.Guarded(wb)
+    outs = [gu.Guarded(2 * count) for _ in range(nranks)]
+    eq.allreduce_sim_bf16([xd[r] for r in range(nranks)], outs, nranks, count, ws, wb, gu.stream_handle())
+    torch.cuda.synchronize()
+    ws.check()
+    exp = oracle.allreduce_bf16(wl.as_u16(x))
+    for r in range(nranks):
+        outs[r].check()
+        gu.assert_same_words(outs[r].view(torch.bfloat16), exp[r], f"bf16 ring output of rank {r}")
+
+
+def test_error_within_bound_on_gpu_outputs(gu):
+    """End-to-end error of the GPU result against the exact fp64 sum stays under the bound
+    accumulated over the hops (bound evaluated by the oracle from the GPU's own trace)."""
+    w = wl.C5
+    count = 64 * 256 * 8
+    x = wl.make_inputs(w, count=count)
+    out, ws = gu.run_sim(x.cuda(), 256, keep_trace=True)
+    sc, _ = eq.trace_views(ws.u8, 64, count, 256, keep_trace=True)
+    bound = oracle.error_bound(sc.cpu().numpy().reshape(64, 64, -1), wl.as_u16(out[0]), 64, 256)
+    exact = x.double().sum(dim=0).numpy()
+    err = np.abs(out[0].double().cpu().numpy() - exact)
+    assert np.all(err <= bound)
+
+
+def test_launch_ranges_compose_to_the_whole_schedule(gu):
+    w = wl.Workload("t", 5, 5 * 256 * 9, 256, "normal", seed=9)
+    x = wl.make_inputs(w).cuda()
+    ref, _ = gu.run_sim(x, 256)
+    wb = eq.allreduce_sim_workspace_bytes(5, w.count, 256, False)
+    ws = gu.Guarded(wb)
+    outs = [gu.Guarded(2 * w.count) for _ in range(5)]
+    ins = [x[r] for r in range(5)]
+    for first, last in ((0, 0), (1, 2), (3, 3), (4, 5)):
+        eq.allreduce_sim_range(ins, outs, 5, w.count, 256, ws, wb, False, first, last, gu.stream_handle())
+    torch.cuda.synchronize()
+    for r in range(5):
+        outs[r].check()
+        assert torch.equal(outs[r].view(torch.int16), ref[r].view(torch.int16))
+    with pytest.raises(eq.EquarxError):
+        eq.allreduce_sim_range(ins, outs, 5, w.count, 256, ws, wb, False, 2, 6, gu.stream_handle())
