@@ -1,0 +1,70 @@
+"""Host logic of bench.py: byte accounting and the multi-replica aggregation
+(two gloo ranks on CPU stand in for two GPUs running independent replicas)."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+import bench  # noqa: E402
+
+
+def test_algorithmic_bytes_match_the_closed_form():
+    # n * N * (6 + 8/B); config 3: N=8, n=8192*5376, B=256 -> 2124.9 MB
+    n, N, B = 8192 * 5376, 8, 256
+    assert bench.algorithmic_bytes(N, n, B) == n * N * (6 + 8 / B)
+    assert round(bench.algorithmic_bytes(N, n, B) / 1e6, 1) == 2124.9
+    total = (bench.launch_bytes("quantize_blocks", N, n, B)
+             + (N - 1) * bench.launch_bytes("rs_step_dequant_add_requant", N, n, B)
+             + bench.launch_bytes("ag_dequant", N, n, B))
+    assert total == bench.algorithmic_bytes(N, n, B)
+
+
+def test_aggregate_value_is_whole_job():
+    # 2 replicas, each reducing 1e9 bytes in 1 ms -> 2000 GB/s
+    assert bench.aggregate_value(1e9, 1.0, 2) == pytest.approx(2000.0)
+
+
+def _worker(rank, world, port, q):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    ms = 1.0 + 2.0 * rank                      # rank 1 is the slow replica
+    got = bench.max_over_ranks(ms, world, torch.device("cpu"))
+    dist.barrier()
+    q.put((rank, got))
+    dist.destroy_process_group()
+
+
+def test_max_over_ranks_two_gloo_processes():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 29500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = dict(q.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert got == {0: 3.0, 1: 3.0}
+
+
+def test_reference_arm_prints_one_line_and_other_ranks_stay_silent():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "3",
+                          "--warmup", "3", "--workload", "C1"], env=env, capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0 and out.stdout.strip() == ""
+    env["RANK"] = "0"
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "3",
+                          "--warmup", "3", "--workload", "C1"], env=env, capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["unit"] == "GB/s" and line["value"] > 0
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
