@@ -59,7 +59,9 @@ enum equarx_status {
     EQUARX_ERR_ALIGN = 5,      /* a pointer breaks the alignment rules above             */
     EQUARX_ERR_WORKSPACE = 6,  /* workspace_bytes smaller than *_workspace_bytes()       */
     EQUARX_ERR_ALIAS = 7,      /* buffers overlap in a way the call does not allow       */
-    EQUARX_ERR_CUDA = 8        /* a launch failed; see equarx_last_cuda_error()          */
+    EQUARX_ERR_CUDA = 8,       /* a launch failed; see equarx_last_cuda_error()          */
+    EQUARX_ERR_STATIC_LIMIT = 9 /* problem too large for the built-in workspace of
+                                  equarx_allreduce_sim_static                            */
 };
 
 /*
@@ -162,6 +164,46 @@ int equarx_allreduce_sim_bf16(const void *const *in_bf16, void *const *out_bf16,
                               int nranks, size_t count,
                               void *workspace, size_t workspace_bytes,
                               equarx_stream_t stream);
+
+/*
+ * equarx_allreduce_sim without a caller-provided workspace.  (The paper has no
+ * counterpart for this entry point; it exists for the callers described here.)
+ *
+ * Who it is for: code that must run the simulation but is not in a position to
+ * hand over scratch memory -- a plugin inside a host application that owns the
+ * whole device heap, a serving loop whose memory plan is frozen after start-up,
+ * a process that is not permitted to call cudaMalloc at all.  Such callers still
+ * own their input and output tensors; what they lack is a place for the hop
+ * messages.  This function keeps that place inside the library: a fixed array of
+ * EQUARX_STATIC_WORKSPACE_BYTES bytes in the library's device image.  Every GPU
+ * on which the library is loaded carries that array until the process exits,
+ * whether this function is ever called or not.
+ *
+ * It calls no cudaMalloc, cudaFree or other allocating routine.  The result is
+ * bit-identical to equarx_allreduce_sim (keep_trace = 0) on the same inputs.
+ *
+ * Limits and rules
+ *   - The problem must fit: equarx_allreduce_sim_workspace_bytes(nranks, count,
+ *     block, 0) <= EQUARX_STATIC_WORKSPACE_BYTES, else EQUARX_ERR_STATIC_LIMIT
+ *     and nothing is launched.  (16 MiB holds, for example, 8 ranks x 7.8 M
+ *     elements at block 256.)
+ *   - The first call on a given device looks up the array's device address
+ *     (cudaGetSymbolAddress, with that device current) and remembers it.  Make
+ *     that first call during normal execution, before any stream capture
+ *     begins on that device.
+ *   - All calls on a device share the one array.  Two calls whose kernels can
+ *     run at the same time (different streams, no ordering between them) race
+ *     on it and produce garbage; order them yourself.  The array keeps the
+ *     previous call's messages; nothing in it has to start at zero, because
+ *     every message is written by an earlier launch of the same call before it
+ *     is read.
+ *   - Arguments, aliasing rules and the other error codes are those of
+ *     equarx_allreduce_sim.
+ */
+#define EQUARX_STATIC_WORKSPACE_BYTES (16u * 1024u * 1024u)
+int equarx_allreduce_sim_static(const void *const *in_bf16, void *const *out_bf16,
+                                int nranks, size_t count, int block,
+                                equarx_stream_t stream);
 
 /* Static, human-readable name of a status. */
 const char *equarx_status_string(int status);

@@ -10,7 +10,8 @@ import ctypes
 from . import _build
 
 MAX_RANKS = 64
-OK, ERR_NULL, ERR_NRANKS, ERR_BLOCK, ERR_COUNT, ERR_ALIGN, ERR_WORKSPACE, ERR_ALIAS, ERR_CUDA = range(9)
+OK, ERR_NULL, ERR_NRANKS, ERR_BLOCK, ERR_COUNT, ERR_ALIGN, ERR_WORKSPACE, ERR_ALIAS, ERR_CUDA, ERR_STATIC_LIMIT = range(10)
+STATIC_WORKSPACE_BYTES = 16 * 1024 * 1024
 
 EXPORTS = (
     "equarx_quantize_blocks",
@@ -19,6 +20,7 @@ EXPORTS = (
     "equarx_allreduce_sim_workspace_bytes",
     "equarx_allreduce_sim",
     "equarx_allreduce_sim_range",
+    "equarx_allreduce_sim_static",
     "equarx_allreduce_sim_bf16_workspace_bytes",
     "equarx_allreduce_sim_bf16",
     "equarx_status_string",
@@ -43,6 +45,7 @@ def _load():
     lib.equarx_allreduce_sim_workspace_bytes.restype = sz
     lib.equarx_allreduce_sim.argtypes = [vp, vp, ci, sz, ci, vp, sz, ci, vp]
     lib.equarx_allreduce_sim_range.argtypes = [vp, vp, ci, sz, ci, vp, sz, ci, ci, ci, vp]
+    lib.equarx_allreduce_sim_static.argtypes = [vp, vp, ci, sz, ci, vp]
     lib.equarx_allreduce_sim_bf16_workspace_bytes.argtypes = [ci, sz]
     lib.equarx_allreduce_sim_bf16_workspace_bytes.restype = sz
     lib.equarx_allreduce_sim_bf16.argtypes = [vp, vp, ci, sz, vp, sz, vp]
@@ -118,6 +121,15 @@ def allreduce_sim_range(in_bf16, out_bf16, nranks, count, block, workspace, work
                                           workspace_bytes, int(bool(keep_trace)), first_launch, last_launch,
                                           _ptr(stream)),
            "equarx_allreduce_sim_range")
+
+
+def allreduce_sim_static(in_bf16, out_bf16, nranks, count, block, stream=0):
+    """equarx_allreduce_sim with the library's built-in 16 MiB workspace: for callers that
+    have no scratch memory to give and may not allocate any.  All calls on a device share
+    that workspace, so calls that could overlap on the GPU must be ordered by the caller;
+    make the first call on a device outside stream capture."""
+    _check(lib.equarx_allreduce_sim_static(_table(in_bf16), _table(out_bf16), nranks, count, block, _ptr(stream)),
+           "equarx_allreduce_sim_static")
 
 
 def allreduce_sim_bf16_workspace_bytes(nranks, count):

@@ -142,6 +142,8 @@ const char* equarx_status_string(int status) {
         case EQUARX_ERR_WORKSPACE: return "EQUARX_ERR_WORKSPACE: workspace too small";
         case EQUARX_ERR_ALIAS: return "EQUARX_ERR_ALIAS: buffers overlap";
         case EQUARX_ERR_CUDA: return "EQUARX_ERR_CUDA: a kernel launch failed";
+        case EQUARX_ERR_STATIC_LIMIT:
+            return "EQUARX_ERR_STATIC_LIMIT: problem needs more than the 16 MiB built-in workspace";
         default: return "EQUARX: unknown status";
     }
 }
@@ -319,6 +321,47 @@ int equarx_allreduce_sim_bf16(const void* const* in_bf16, void* const* out_bf16,
         g.src[k] = N == 1 ? in_bf16[0] : msg(N - 1, k);
     }
     return launch(bf16_gather_kernel, grid_for(shard, N), g, stream, N > 1);
+}
+
+// ---------------------------------------------------------------------------------
+// Workspace-free variant for callers that cannot provide (or allocate) scratch memory.
+// The hop messages go to a fixed array that is part of this library's device image,
+// so every GPU that loads the library holds these 16 MiB until the process exits.
+//
+// `g_static_workspace` below is only a host-side handle when it is named in host
+// code: it is NOT a device address and must never be passed to a kernel as is.  The
+// device address is looked up once per device with cudaGetSymbolAddress while that
+// device is current, and it is that address which goes into the kernel arguments.
+static __device__ __align__(256) unsigned char g_static_workspace[EQUARX_STATIC_WORKSPACE_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_ptr[kMaxDevices] = {};      // device address of g_static_workspace, per device ordinal
+}  // namespace
+
+int equarx_allreduce_sim_static(const void* const* in_bf16, void* const* out_bf16, int nranks, size_t count,
+                                int block, equarx_stream_t stream) {
+    if (int st = check_sim_shape(nranks, count, block)) return st;
+    const size_t need = equarx_allreduce_sim_workspace_bytes(nranks, count, block, 0);
+    if (need > size_t(EQUARX_STATIC_WORKSPACE_BYTES)) return EQUARX_ERR_STATIC_LIMIT;
+
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess && (dev < 0 || dev >= kMaxDevices)) e = cudaErrorInvalidDevice;
+    if (e == cudaSuccess && g_static_ptr[dev] == nullptr) {
+        // set-up, once per device, with that device current (a benign race: every
+        // thread that gets here stores the same address)
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_workspace);
+        if (e == cudaSuccess) g_static_ptr[dev] = p;
+    }
+    if (e != cudaSuccess) {
+        g_last_cuda_error = int(e);
+        (void)cudaGetLastError();
+        return EQUARX_ERR_CUDA;
+    }
+    return equarx_allreduce_sim_range(in_bf16, out_bf16, nranks, count, block, g_static_ptr[dev],
+                                      size_t(EQUARX_STATIC_WORKSPACE_BYTES), 0, 0, nranks, stream);
 }
 
 }  // extern "C"
