@@ -41,10 +41,14 @@ DAR_TRAFFIC_BYTES_PER_ELEMENT = 3.017
 
 
 def workload_by_name(name):
+    """C1 | C2 | C3 | C5, or a point of the message-size sweep: sweep:<nranks>:<bytes per rank>:<block>:<dist>."""
     from paper_2506_17615_b200 import workloads as wl
+    if name.startswith("sweep:"):
+        _, n, nbytes, block, dist = name.split(":")
+        return wl.sweep_point(int(n), int(nbytes), int(block), dist)
     table = {"C1": wl.C1, "C2": wl.C2, "C3": wl.C3, "C5": wl.C5}
     if name not in table:
-        raise SystemExit(f"unknown workload {name}; choose from {sorted(table)}")
+        raise SystemExit(f"unknown workload {name}; choose from {sorted(table)} or sweep:N:bytes:block:dist")
     return table[name]
 
 

@@ -18,8 +18,8 @@
  *     may be freed as soon as it returns.  All other pointers are DEVICE
  *     pointers.
  *   - bf16 tensors are raw 16-bit words; bf16 buffers must be 32-byte
- *     aligned (they are moved with 256-bit accesses), int8 code buffers and
- *     workspaces 16-byte aligned, scale buffers 4-byte aligned.
+ *     aligned (they are moved with 256-bit accesses) and so must workspaces;
+ *     int8 code buffers 16-byte aligned, scale buffers 4-byte aligned.
  *   - `block` is the number of contiguous elements that share one fp32
  *     scale (Section 3.2, Fig. 3: one scale factor per block of entries);
  *     supported values 64, 128, 256, 512.
@@ -102,14 +102,19 @@ int equarx_ag_dequant(const int8_t *codes, const float *scales, size_t count, in
 
 /*
  * Bytes of workspace equarx_allreduce_sim needs; 0 if the arguments are
- * invalid.  Layout, with shard = count/nranks, bps = shard/block and
- * slots = keep_trace ? nranks*nranks : 2*nranks:
- *   float  scales[slots][bps]    at offset 0
- *   int8_t codes [slots][shard]  at offset round_up(4*slots*bps, 256)
- * Without trace the slot of rank r's message at ring step s is (s&1)*nranks+r
- * (ping-pong).  With trace the slot of shard k's event j (the message sent at
- * step j by rank (k+1+j) mod nranks; event nranks-1 is the all-gather
- * message) is k*nranks+j, and every message of the run is kept.
+ * invalid.  The workspace holds messages.  A message (one shard's codes and
+ * scales) is stored as a sequence of 544-byte records, one per tile of 512
+ * consecutive elements of the shard: first 8 floats of metadata (the tile's
+ * 512/block scales in order, then zeros), then the tile's 512 int8 codes
+ * ("send the metadata before any microshards", Section 3.1).  The last record
+ * of a message is only partly used if the shard is not a multiple of 512.
+ * A message slot is tiles = ceil(shard/512) records; slot i starts at byte
+ * i*tiles*544.  "Event j of shard k" is the message sent at ring step j by rank
+ * (k+1+j) mod nranks; event nranks-1 is the all-gather message.  Without trace
+ * there are 2*nranks slots and the event's slot is 2*k + (j&1) (ping-pong per
+ * shard: on return the workspace holds the last two events of every shard).
+ * With trace there are nranks*nranks slots, the event's slot is k*nranks + j
+ * and every message of the run is kept.
  */
 size_t equarx_allreduce_sim_workspace_bytes(int nranks, size_t count, int block, int keep_trace);
 
@@ -150,6 +155,31 @@ int equarx_allreduce_sim_range(const void *const *in_bf16, void *const *out_bf16
                                void *workspace, size_t workspace_bytes, int keep_trace,
                                int first_launch, int last_launch, equarx_stream_t stream);
 
+/*
+ * The same AllReduce as ONE persistent launch in deep-pipelined order.  Section
+ * 3.1 splits a shard into microshards that move through the ring steps
+ * independently of one another; here a microshard is a tile of 512 elements
+ * and one warp carries it through all nranks steps and the all-gather without
+ * waiting for the rest of the shard.  Every hop message is still written to
+ * memory as a record and read back from there (by the neighbouring lane, acting
+ * for the receiving rank), but it is consumed right after it was produced and is
+ * therefore served from L2 instead of HBM.  Outputs, and with keep_trace the
+ * whole trace, are identical to equarx_allreduce_sim bit for bit; only the order
+ * in which tiles advance differs.
+ *
+ * Workspace: with keep_trace, the trace exactly as equarx_allreduce_sim lays it
+ * out.  Without, EQUARX_PIPELINE_FIFO_BYTES of staging space: every warp owns a
+ * two-record FIFO that it reuses for all steps of all its tiles (the way a ring
+ * channel reuses its staging buffers); its contents on return are meaningless.
+ * All other arguments and rules as for equarx_allreduce_sim.
+ */
+#define EQUARX_PIPELINE_FIFO_BYTES (8u * 1024u * 1024u)
+size_t equarx_allreduce_sim_pipelined_workspace_bytes(int nranks, size_t count, int block, int keep_trace);
+int equarx_allreduce_sim_pipelined(const void *const *in_bf16, void *const *out_bf16,
+                                   int nranks, size_t count, int block,
+                                   void *workspace, size_t workspace_bytes, int keep_trace,
+                                   equarx_stream_t stream);
+
 /* Workspace bytes of the unquantized comparator (two generations of bf16 messages: 4*count); 0 if invalid. */
 size_t equarx_allreduce_sim_bf16_workspace_bytes(int nranks, size_t count);
 
@@ -185,8 +215,8 @@ int equarx_allreduce_sim_bf16(const void *const *in_bf16, void *const *out_bf16,
  * Limits and rules
  *   - The problem must fit: equarx_allreduce_sim_workspace_bytes(nranks, count,
  *     block, 0) <= EQUARX_STATIC_WORKSPACE_BYTES, else EQUARX_ERR_STATIC_LIMIT
- *     and nothing is launched.  (16 MiB holds, for example, 8 ranks x 7.8 M
- *     elements at block 256.)
+ *     and nothing is launched.  (16 MiB holds, for example, 8 ranks x 7.86 M
+ *     elements: 2*8 message slots of 1920 records.)
  *   - The first call on a given device looks up the array's device address
  *     (cudaGetSymbolAddress, with that device current) and remembers it.  Make
  *     that first call during normal execution, before any stream capture

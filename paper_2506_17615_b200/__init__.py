@@ -12,6 +12,8 @@ from .binding import (  # noqa: F401
     allreduce_sim,
     allreduce_sim_bf16,
     allreduce_sim_bf16_workspace_bytes,
+    allreduce_sim_pipelined,
+    allreduce_sim_pipelined_workspace_bytes,
     allreduce_sim_range,
     allreduce_sim_static,
     allreduce_sim_workspace_bytes,

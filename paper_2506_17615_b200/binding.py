@@ -19,6 +19,8 @@ EXPORTS = (
     "equarx_ag_dequant",
     "equarx_allreduce_sim_workspace_bytes",
     "equarx_allreduce_sim",
+    "equarx_allreduce_sim_pipelined",
+    "equarx_allreduce_sim_pipelined_workspace_bytes",
     "equarx_allreduce_sim_range",
     "equarx_allreduce_sim_static",
     "equarx_allreduce_sim_bf16_workspace_bytes",
@@ -45,6 +47,9 @@ def _load():
     lib.equarx_allreduce_sim_workspace_bytes.restype = sz
     lib.equarx_allreduce_sim.argtypes = [vp, vp, ci, sz, ci, vp, sz, ci, vp]
     lib.equarx_allreduce_sim_range.argtypes = [vp, vp, ci, sz, ci, vp, sz, ci, ci, ci, vp]
+    lib.equarx_allreduce_sim_pipelined.argtypes = [vp, vp, ci, sz, ci, vp, sz, ci, vp]
+    lib.equarx_allreduce_sim_pipelined_workspace_bytes.argtypes = [ci, sz, ci, ci]
+    lib.equarx_allreduce_sim_pipelined_workspace_bytes.restype = sz
     lib.equarx_allreduce_sim_static.argtypes = [vp, vp, ci, sz, ci, vp]
     lib.equarx_allreduce_sim_bf16_workspace_bytes.argtypes = [ci, sz]
     lib.equarx_allreduce_sim_bf16_workspace_bytes.restype = sz
@@ -115,6 +120,17 @@ def allreduce_sim(in_bf16, out_bf16, nranks, count, block, workspace, workspace_
            "equarx_allreduce_sim")
 
 
+def allreduce_sim_pipelined_workspace_bytes(nranks, count, block, keep_trace=False):
+    return lib.equarx_allreduce_sim_pipelined_workspace_bytes(nranks, count, block, int(bool(keep_trace)))
+
+
+def allreduce_sim_pipelined(in_bf16, out_bf16, nranks, count, block, workspace, workspace_bytes, keep_trace=False,
+                            stream=0):
+    _check(lib.equarx_allreduce_sim_pipelined(_table(in_bf16), _table(out_bf16), nranks, count, block,
+                                              _ptr(workspace), workspace_bytes, int(bool(keep_trace)), _ptr(stream)),
+           "equarx_allreduce_sim_pipelined")
+
+
 def allreduce_sim_range(in_bf16, out_bf16, nranks, count, block, workspace, workspace_bytes, keep_trace,
                         first_launch, last_launch, stream=0):
     _check(lib.equarx_allreduce_sim_range(_table(in_bf16), _table(out_bf16), nranks, count, block, _ptr(workspace),
@@ -142,22 +158,32 @@ def allreduce_sim_bf16(in_bf16, out_bf16, nranks, count, workspace, workspace_by
            "equarx_allreduce_sim_bf16")
 
 
-def trace_views(workspace_u8, nranks, count, block, keep_trace=True):
-    """Split a workspace (1-D uint8 tensor or numpy array) into (scales, codes) views.
+RECORD_BYTES, RECORD_HEADER, TILE_ELEMS = 544, 32, 512
+PIPELINE_FIFO_BYTES = 8 * 1024 * 1024
 
-    Returns (float32 [slots, bps], int8 [slots, shard]) with slots = N*N for a
-    trace ([shard k][event j] flattened) or 2*N for the ping-pong layout.
+
+def trace_views(workspace_u8, nranks, count, block, keep_trace=True):
+    """Unpack a message workspace (1-D uint8 torch tensor or numpy array) into
+    (scales float32 [slots, blocks per shard], codes int8 [slots, shard]) copies.
+
+    slots = N*N for a trace (slot k*N + j = event j of shard k) or 2*N for the ping-pong
+    layout (slot 2*k + (j&1)).  The workspace stores 544-byte records: 8 floats of metadata,
+    then 512 codes, one record per 512-element tile of a message.
     """
     shard = count // nranks
     bps = shard // block
+    tiles = (shard + TILE_ELEMS - 1) // TILE_ELEMS
     slots = nranks * nranks if keep_trace else 2 * nranks
-    off = (4 * slots * bps + 255) // 256 * 256
+    per_tile = TILE_ELEMS // block
+    rec = workspace_u8[:slots * tiles * RECORD_BYTES].reshape(slots, tiles, RECORD_BYTES)
     if hasattr(workspace_u8, "numpy"):      # torch tensor
         import torch
-        sc = workspace_u8[:4 * slots * bps].view(torch.float32).view(slots, bps)
-        co = workspace_u8[off:off + slots * shard].view(torch.int8).view(slots, shard)
-        return sc, co
+        hdr = rec[:, :, :RECORD_HEADER].contiguous().view(torch.float32)
+        sc = hdr[:, :, :per_tile].reshape(slots, tiles * per_tile)[:, :bps].contiguous()
+        co = rec[:, :, RECORD_HEADER:].contiguous().view(torch.int8).reshape(slots, tiles * TILE_ELEMS)[:, :shard]
+        return sc, co.contiguous()
     import numpy as np
-    sc = workspace_u8[:4 * slots * bps].view(np.float32).reshape(slots, bps)
-    co = workspace_u8[off:off + slots * shard].view(np.int8).reshape(slots, shard)
-    return sc, co
+    hdr = np.ascontiguousarray(rec[:, :, :RECORD_HEADER]).view(np.float32)
+    sc = np.ascontiguousarray(hdr[:, :, :per_tile].reshape(slots, tiles * per_tile)[:, :bps])
+    co = np.ascontiguousarray(rec[:, :, RECORD_HEADER:]).view(np.int8).reshape(slots, tiles * TILE_ELEMS)[:, :shard]
+    return sc, np.ascontiguousarray(co)

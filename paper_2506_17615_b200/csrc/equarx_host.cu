@@ -85,26 +85,30 @@ inline dim3 grid_for(uint64_t shard, unsigned y) {
     return dim3(unsigned((groups + kThreads - 1) / kThreads), y, 1);
 }
 
-template <bool FIRST>
+template <bool FIRST, bool RECORDS>
 int launch_step(int block, const StepArgs& a, unsigned nranks, cudaStream_t stream, bool dependent) {
     const dim3 grid = grid_for(a.shard, nranks);
     switch (block) {
-        case 64: return launch(rs_step_kernel<4, FIRST>, grid, a, stream, dependent);
-        case 128: return launch(rs_step_kernel<8, FIRST>, grid, a, stream, dependent);
-        case 256: return launch(rs_step_kernel<16, FIRST>, grid, a, stream, dependent);
-        default: return launch(rs_step_kernel<32, FIRST>, grid, a, stream, dependent);
+        case 64: return launch(rs_step_kernel<4, FIRST, RECORDS>, grid, a, stream, dependent);
+        case 128: return launch(rs_step_kernel<8, FIRST, RECORDS>, grid, a, stream, dependent);
+        case 256: return launch(rs_step_kernel<16, FIRST, RECORDS>, grid, a, stream, dependent);
+        default: return launch(rs_step_kernel<32, FIRST, RECORDS>, grid, a, stream, dependent);
     }
 }
 
+template <bool RECORDS>
 int launch_gather(int block, const GatherArgs& a, cudaStream_t stream, bool dependent) {
     const dim3 grid = grid_for(a.shard, a.nranks);
     switch (block) {
-        case 64: return launch(ag_dequant_kernel<4>, grid, a, stream, dependent);
-        case 128: return launch(ag_dequant_kernel<8>, grid, a, stream, dependent);
-        case 256: return launch(ag_dequant_kernel<16>, grid, a, stream, dependent);
-        default: return launch(ag_dequant_kernel<32>, grid, a, stream, dependent);
+        case 64: return launch(ag_dequant_kernel<4, RECORDS>, grid, a, stream, dependent);
+        case 128: return launch(ag_dequant_kernel<8, RECORDS>, grid, a, stream, dependent);
+        case 256: return launch(ag_dequant_kernel<16, RECORDS>, grid, a, stream, dependent);
+        default: return launch(ag_dequant_kernel<32, RECORDS>, grid, a, stream, dependent);
     }
 }
+
+// bytes of one message slot in the record layout: one 544-byte record per 512-element tile
+inline size_t slot_bytes(size_t shard) { return (shard + kTileElems - 1) / kTileElems * size_t(kRecordBytes); }
 
 // in/out tables of a simulation: NULLs, alignment, overlap.  out[r] == in[r] is the
 // one overlap allowed.
@@ -164,7 +168,7 @@ int equarx_quantize_blocks(const void* x_bf16, size_t count, int block, int8_t* 
     a.scales_out = scales;
     a.shard = count;
     a.bps = count / size_t(block);
-    return launch_step<true>(block, a, 1, stream, false);
+    return launch_step<true, false>(block, a, 1, stream, false);
 }
 
 int equarx_rs_step_dequant_add_requant(const int8_t* codes_in, const float* scales_in, const void* local_bf16,
@@ -189,7 +193,7 @@ int equarx_rs_step_dequant_add_requant(const int8_t* codes_in, const float* scal
     a.scales_out = scales_out;
     a.shard = count;
     a.bps = count / size_t(block);
-    return launch_step<false>(block, a, 1, stream, false);
+    return launch_step<false, false>(block, a, 1, stream, false);
 }
 
 int equarx_ag_dequant(const int8_t* codes, const float* scales, size_t count, int block, void* out_bf16,
@@ -206,14 +210,14 @@ int equarx_ag_dequant(const int8_t* codes, const float* scales, size_t count, in
     a.shard = count;
     a.bps = count / size_t(block);
     a.nranks = 1;
-    return launch_gather(block, a, stream, false);
+    return launch_gather<false>(block, a, stream, false);
 }
 
 size_t equarx_allreduce_sim_workspace_bytes(int nranks, size_t count, int block, int keep_trace) {
     if (check_sim_shape(nranks, count, block) != EQUARX_OK) return 0;
-    const size_t N = size_t(nranks), shard = count / N, bps = shard / size_t(block);
+    const size_t N = size_t(nranks);
     const size_t slots = keep_trace ? N * N : 2 * N;
-    return round_up(4 * slots * bps, 256) + slots * shard;
+    return slots * slot_bytes(count / N);
 }
 
 int equarx_allreduce_sim(const void* const* in_bf16, void* const* out_bf16, int nranks, size_t count, int block,
@@ -230,28 +234,24 @@ int equarx_allreduce_sim_range(const void* const* in_bf16, void* const* out_bf16
     if (!workspace) return EQUARX_ERR_NULL;
     const size_t need = equarx_allreduce_sim_workspace_bytes(nranks, count, block, keep_trace);
     if (workspace_bytes < need) return EQUARX_ERR_WORKSPACE;
-    if (!aligned(workspace, 16)) return EQUARX_ERR_ALIGN;
+    if (!aligned(workspace, 32)) return EQUARX_ERR_ALIGN;
     if (int st = check_tables(in_bf16, out_bf16, nranks, 2 * count, workspace, need)) return st;
 
     const uint32_t N = uint32_t(nranks);
-    const size_t shard = count / N, bps = shard / size_t(block);
-    const size_t slots = keep_trace ? size_t(N) * N : 2 * size_t(N);
-    float* scales = static_cast<float*>(workspace);
-    int8_t* codes = static_cast<int8_t*>(workspace) + round_up(4 * slots * bps, 256);
+    const size_t shard = count / N;
+    int8_t* records = static_cast<int8_t*>(workspace);
 
     // shard that rank r sends at step s, and where that message is kept
     auto shard_of = [N](uint32_t s, uint32_t r) { return (r + 2 * N - 1 - s % N) % N; };
     auto slot_of = [&](uint32_t s, uint32_t r) {
-        return keep_trace ? shard_of(s, r) * N + s : (s & 1u) * N + r;
+        return keep_trace ? shard_of(s, r) * N + s : shard_of(s, r) * 2 + (s & 1u);
     };
 
     StepArgs a = {};
-    a.codes_in = codes;
-    a.scales_in = scales;
-    a.codes_out = codes;
-    a.scales_out = scales;
+    a.codes_in = records;
+    a.codes_out = records;
     a.shard = shard;
-    a.bps = bps;
+    a.bps = slot_bytes(shard);
     const uint32_t first = uint32_t(first_launch), last = uint32_t(last_launch);
     for (uint32_t s = first; s < N && s <= last; ++s) {
         for (uint32_t r = 0; r < N; ++r) {
@@ -260,8 +260,8 @@ int equarx_allreduce_sim_range(const void* const* in_bf16, void* const* out_bf16
             a.in_slot[r] = s ? slot_of(s - 1, (r + N - 1) % N) : 0;
         }
         // only a launch that follows another launch of this call may overlap its predecessor
-        const int st = s == 0 ? launch_step<true>(block, a, N, stream, false)
-                              : launch_step<false>(block, a, N, stream, s > first);
+        const int st = s == 0 ? launch_step<true, true>(block, a, N, stream, false)
+                              : launch_step<false, true>(block, a, N, stream, s > first);
         if (st) return st;
     }
     if (last < N) return EQUARX_OK;
@@ -271,12 +271,86 @@ int equarx_allreduce_sim_range(const void* const* in_bf16, void* const* out_bf16
         g.out[k] = out_bf16[k];
         g.slot[k] = slot_of(N - 1, k);     // after step N-1 rank k holds shard k
     }
-    g.codes = codes;
-    g.scales = scales;
+    g.codes = records;
     g.shard = shard;
-    g.bps = bps;
+    g.bps = slot_bytes(shard);
     g.nranks = N;
-    return launch_gather(block, g, stream, first < N);
+    return launch_gather<true>(block, g, stream, first < N);
+}
+
+size_t equarx_allreduce_sim_pipelined_workspace_bytes(int nranks, size_t count, int block, int keep_trace) {
+    if (check_sim_shape(nranks, count, block) != EQUARX_OK) return 0;
+    if (keep_trace) return equarx_allreduce_sim_workspace_bytes(nranks, count, block, 1);
+    return size_t(EQUARX_PIPELINE_FIFO_BYTES);
+}
+
+int equarx_allreduce_sim_pipelined(const void* const* in_bf16, void* const* out_bf16, int nranks, size_t count,
+                                   int block, void* workspace, size_t workspace_bytes, int keep_trace,
+                                   equarx_stream_t stream) {
+    if (int st = check_sim_shape(nranks, count, block)) return st;
+    if (!workspace) return EQUARX_ERR_NULL;
+    const size_t need = equarx_allreduce_sim_pipelined_workspace_bytes(nranks, count, block, keep_trace);
+    if (workspace_bytes < need) return EQUARX_ERR_WORKSPACE;
+    if (!aligned(workspace, 32)) return EQUARX_ERR_ALIGN;
+    if (int st = check_tables(in_bf16, out_bf16, nranks, 2 * count, workspace, need)) return st;
+
+    const uint32_t N = uint32_t(nranks);
+    const size_t shard = count / N;
+    PipeArgs a = {};
+    for (uint32_t r = 0; r < N; ++r) {
+        a.in[r] = in_bf16[r];
+        a.out[r] = out_bf16[r];
+    }
+    a.records = static_cast<char*>(workspace);
+    a.shard = shard;
+    a.tiles_per_shard = (shard + kTileElems - 1) / kTileElems;
+    a.nranks = N;
+    a.keep_trace = keep_trace ? 1u : 0u;
+
+    const void* kernel = nullptr;
+    switch (block) {
+        case 64: kernel = reinterpret_cast<const void*>(pipelined_kernel<4>); break;
+        case 128: kernel = reinterpret_cast<const void*>(pipelined_kernel<8>); break;
+        case 256: kernel = reinterpret_cast<const void*>(pipelined_kernel<16>); break;
+        default: kernel = reinterpret_cast<const void*>(pipelined_kernel<32>); break;
+    }
+    // persistent grid: a whole number of CTAs per SM, chosen so that the warp tiles split
+    // into full rounds as evenly as possible
+    int dev = 0, sms = 0, occ = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kPipeThreads, 0);
+    if (e != cudaSuccess || sms < 1 || occ < 1) {
+        g_last_cuda_error = int(e);
+        (void)cudaGetLastError();
+        return EQUARX_ERR_CUDA;
+    }
+    const uint64_t tiles = a.tiles_per_shard * N, wpc = kPipeThreads / 32;
+    uint64_t best_ctas = 0;
+    double best_eff = -1.0;
+    for (int c = occ; c >= (occ + 1) / 2; --c) {
+        const uint64_t ctas = uint64_t(sms) * c, w = ctas * wpc;
+        const uint64_t rounds = (tiles + w - 1) / w;
+        const double eff = double(tiles) / double(rounds * w);
+        if (eff > best_eff + 1e-9) {
+            best_eff = eff;
+            best_ctas = ctas;
+        }
+    }
+    const uint64_t max_needed = (tiles + wpc - 1) / wpc;
+    if (best_ctas > max_needed) best_ctas = max_needed;
+    // every warp owns a two-record staging FIFO in the workspace
+    const uint64_t fifo_ctas = uint64_t(EQUARX_PIPELINE_FIFO_BYTES) / (2 * kRecordBytes) / wpc;
+    if (!keep_trace && best_ctas > fifo_ctas) best_ctas = fifo_ctas;
+
+    void* params[1] = {&a};
+    e = cudaLaunchKernel(kernel, dim3(unsigned(best_ctas)), dim3(kPipeThreads), params, 0, stream);
+    if (e != cudaSuccess) {
+        g_last_cuda_error = int(e);
+        (void)cudaGetLastError();
+        return EQUARX_ERR_CUDA;
+    }
+    return EQUARX_OK;
 }
 
 size_t equarx_allreduce_sim_bf16_workspace_bytes(int nranks, size_t count) {

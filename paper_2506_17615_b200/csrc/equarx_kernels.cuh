@@ -80,6 +80,44 @@ __device__ __forceinline__ void st_scale(float* p, float v, uint64_t pol) {
     asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(p), "f"(v), "l"(pol) : "memory");
 }
 
+// Accessors for data that is written and read inside the SAME launch (the pipelined
+// kernel): no read-only (.nc) path, L2 only.
+__device__ __forceinline__ Vec8 ld_coherent_256(const void* p) {
+    Vec8 r;
+    asm volatile(
+        "ld.global.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+        : "=r"(r.w[0]), "=r"(r.w[1]), "=r"(r.w[2]), "=r"(r.w[3]),
+          "=r"(r.w[4]), "=r"(r.w[5]), "=r"(r.w[6]), "=r"(r.w[7])
+        : "l"(p)
+        : "memory");
+    return r;
+}
+
+__device__ __forceinline__ uint4 ld_coherent_128(const void* p) {
+    uint4 r;
+    asm volatile("ld.global.cg.v4.b32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p)
+                 : "memory");
+    return r;
+}
+
+__device__ __forceinline__ float ld_coherent_f32(const float* p) {
+    float r;
+    asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(r) : "l"(p) : "memory");
+    return r;
+}
+
+__device__ __forceinline__ void st_plain_128(void* p, const uint4& r) {
+    asm volatile("st.global.cg.v4.b32 [%0], {%1,%2,%3,%4};"
+                 ::"l"(p), "r"(r.x), "r"(r.y), "r"(r.z), "r"(r.w)
+                 : "memory");
+}
+
+__device__ __forceinline__ void st_plain_f32(float* p, float v) {
+    asm volatile("st.global.cg.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
+}
+
 // Programmatic dependent launch: let the next step's CTAs be scheduled while this
 // grid drains, and order this grid's dependent reads/writes after the previous grid.
 __device__ __forceinline__ void pdl_launch_dependents() {
@@ -120,24 +158,35 @@ __device__ __forceinline__ float block_max(float m) {
     return m;
 }
 
+// 3-input max (sm_100): halves the instruction count of the in-lane max.
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 // Q_p1 + Q_p2 on the 16 values of one lane; the block is LPB neighbouring lanes.
 // |v * inv| <= 127 * (1 + 2^-24)^2 < 127.5, so the rounded code never leaves
 // [-127, 127] and needs no clamp; adding 1.5 * 2^23 rounds to nearest-even on the
 // integer grid and leaves the two's-complement code in the low byte.
+// Each lane performs ONE of the block's two IEEE divisions (even lanes amax/127, odd
+// lanes 127/amax; the operands are selected, the instruction stream is the same) and
+// the pair of lanes exchanges the quotients with two shuffles.
 template <int LPB>
 __device__ __forceinline__ void quantize_lane(const float (&v)[16], uint4& codes, float& scale) {
-    float m = 0.0f;
-#pragma unroll
-    for (int i = 0; i < 16; ++i) m = fmaxf(m, fabsf(v[i]));
+    float m = max3(fabsf(v[0]), fabsf(v[1]), fabsf(v[2]));
+    float m1 = max3(fabsf(v[3]), fabsf(v[4]), fabsf(v[5]));
+    float m2 = max3(fabsf(v[6]), fabsf(v[7]), fabsf(v[8]));
+    float m3 = max3(fabsf(v[9]), fabsf(v[10]), fabsf(v[11]));
+    m = max3(m, fabsf(v[12]), fabsf(v[13]));
+    m1 = max3(m1, fabsf(v[14]), fabsf(v[15]));
+    m = max3(m, m1, fmaxf(m2, m3));
     m = block_max<LPB>(m);
-    float inv;
-    if (m >= 0x1p-118f) {
-        scale = __fdiv_rn(m, 127.0f);
-        inv = __fdiv_rn(127.0f, m);
-    } else {
-        scale = 0.0f;
-        inv = 0.0f;
-    }
+    const bool odd = threadIdx.x & 1u;
+    const float quot = __fdiv_rn(odd ? 127.0f : m, odd ? m : 127.0f);
+    const float keep = m >= 0x1p-118f ? quot : 0.0f;      // flush rule: scale = inv = 0
+    scale = __shfl_sync(0xFFFFFFFFu, keep, (threadIdx.x & 30u));
+    const float inv = __shfl_sync(0xFFFFFFFFu, keep, (threadIdx.x & 30u) | 1u);
     uint32_t b[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i)
@@ -158,19 +207,39 @@ __device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
     return d;
 }
 
+// ---------------------------------------------------------------- message layouts
+// SPLIT   (the per-step entry points): codes[count] and scales[count/B] are separate arrays.
+// RECORDS (the simulations): a message is a sequence of 544-byte records, one per tile of
+//         512 elements: 8 floats of metadata first (the tile's 512/B scales, zero padded to
+//         one 32-byte sector), then the 512 codes ("send the metadata before any
+//         microshards", Section 3.1).  Every sector of a record is written whole, so a
+//         message that is read back while it is still in L2 never needs a fill from DRAM.
+constexpr int kTileElems = 512;
+constexpr int kRecordHeader = 32;
+constexpr int kRecordBytes = kRecordHeader + kTileElems;
+
+template <int LPB>
+__device__ __forceinline__ void st_record(char* rec, uint32_t lane, bool lane_active, bool tile_active,
+                                          const uint4& codes, float scale, uint64_t pol) {
+    // lanes 0..7 write the header sector: lane i holds the scale of block i of the tile
+    float hdr = __shfl_sync(0xFFFFFFFFu, scale, (lane * LPB) & 31u);
+    if (lane >= 32u / LPB) hdr = 0.0f;
+    if (tile_active && lane < 8) st_scale(reinterpret_cast<float*>(rec) + lane, hdr, pol);
+    if (lane_active) st_wire_128(rec + kRecordHeader + lane * 16, codes, pol);
+}
+
 // ---------------------------------------------------------------- kernel arguments
-// One launch covers every simulated rank.  Messages live in "slots" of a scales
-// region and a codes region (slot * bps floats, slot * shard bytes).
+// One launch covers every simulated rank.  Messages live in "slots".
 struct StepArgs {
     const void* x[kMaxRanks];        // rank r's bf16 shard for this step
     uint32_t in_slot[kMaxRanks];     // message received by rank r (unused at step 0)
     uint32_t out_slot[kMaxRanks];    // message produced by rank r
-    const int8_t* codes_in;
-    const float* scales_in;
+    const int8_t* codes_in;          // SPLIT: codes region; RECORDS: record region
+    const float* scales_in;          // SPLIT only
     int8_t* codes_out;
     float* scales_out;
     uint64_t shard;                  // elements per message
-    uint64_t bps;                    // blocks per message
+    uint64_t bps;                    // SPLIT: blocks per message; RECORDS: bytes per slot
 };
 
 struct GatherArgs {
@@ -179,8 +248,18 @@ struct GatherArgs {
     const int8_t* codes;
     const float* scales;
     uint64_t shard;
-    uint64_t bps;
+    uint64_t bps;                    // as in StepArgs
     uint32_t nranks;
+};
+
+struct PipeArgs {
+    const void* in[kMaxRanks];       // input tensor of rank r (whole tensor)
+    void* out[kMaxRanks];            // output tensor of rank r
+    char* records;                   // trace: record region [shard k][event j][tile]; else per-warp FIFOs
+    uint64_t shard;
+    uint64_t tiles_per_shard;        // 512-element tiles per shard (the last one may be ragged)
+    uint32_t nranks;
+    uint32_t keep_trace;
 };
 
 struct Bf16StepArgs {
@@ -201,11 +280,13 @@ struct Bf16GatherArgs {
 // Ring step: FIRST = step 0 (quantize only), else dequantize-add-requantize.
 // Step 0 is never launched as a programmatic dependent: it reads tensors that an
 // earlier in-place all-gather on the same stream may still be writing.
-template <int LPB, bool FIRST>
+template <int LPB, bool FIRST, bool RECORDS>
 __global__ void __launch_bounds__(kThreads) rs_step_kernel(const __grid_constant__ StepArgs a) {
     const uint32_t r = blockIdx.y;
+    const uint32_t lane = threadIdx.x & 31u;
     const uint64_t g = (uint64_t)blockIdx.x * kThreads + threadIdx.x;   // 16-element group
-    const bool active = g < (a.shard >> 4);
+    const uint64_t groups = a.shard >> 4;
+    const bool active = g < groups;
     const uint64_t pol = policy_keep();
 
     Vec8 xw = {};
@@ -220,8 +301,14 @@ __global__ void __launch_bounds__(kThreads) rs_step_kernel(const __grid_constant
         float s = 0.0f;
         if (active) {
             const uint64_t slot = a.in_slot[r];
-            c = ld_wire_128(a.codes_in + slot * a.shard + g * 16, pol);
-            s = ld_scale(a.scales_in + slot * a.bps + g / LPB, pol);
+            if (RECORDS) {
+                const char* rec = reinterpret_cast<const char*>(a.codes_in) + slot * a.bps + (g >> 5) * kRecordBytes;
+                c = ld_wire_128(rec + kRecordHeader + lane * 16, pol);
+                s = ld_scale(reinterpret_cast<const float*>(rec) + lane / LPB, pol);
+            } else {
+                c = ld_wire_128(a.codes_in + slot * a.shard + g * 16, pol);
+                s = ld_scale(a.scales_in + slot * a.bps + g / LPB, pol);
+            }
         }
         float q[16];
         codes_to_f32x16(c, q);
@@ -232,17 +319,21 @@ __global__ void __launch_bounds__(kThreads) rs_step_kernel(const __grid_constant
     uint4 codes;
     float scale;
     quantize_lane<LPB>(v, codes, scale);
-    if (active) {
-        const uint64_t slot = a.out_slot[r];
+    const uint64_t slot = a.out_slot[r];
+    if (RECORDS) {
+        char* rec = reinterpret_cast<char*>(a.codes_out) + slot * a.bps + (g >> 5) * kRecordBytes;
+        st_record<LPB>(rec, lane, active, (g - lane) < groups, codes, scale, pol);
+    } else if (active) {
         st_wire_128(a.codes_out + slot * a.shard + g * 16, codes, pol);
         if ((threadIdx.x & (LPB - 1)) == 0) st_scale(a.scales_out + slot * a.bps + g / LPB, scale, pol);
     }
 }
 
 // All-gather receive side: one read of shard k's final message, nranks bf16 writes.
-template <int LPB>
+template <int LPB, bool RECORDS>
 __global__ void __launch_bounds__(kThreads) ag_dequant_kernel(const __grid_constant__ GatherArgs a) {
     const uint32_t k = blockIdx.y;
+    const uint32_t lane = threadIdx.x & 31u;
     const uint64_t g = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
     const bool active = g < (a.shard >> 4);
     const uint64_t pol = policy_keep();
@@ -250,8 +341,16 @@ __global__ void __launch_bounds__(kThreads) ag_dequant_kernel(const __grid_const
     pdl_wait_prior_grid();
     if (!active) return;
     const uint64_t slot = a.slot[k];
-    const uint4 c = ld_wire_128(a.codes + slot * a.shard + g * 16, pol);
-    const float s = ld_scale(a.scales + slot * a.bps + g / LPB, pol);
+    uint4 c;
+    float s;
+    if (RECORDS) {
+        const char* rec = reinterpret_cast<const char*>(a.codes) + slot * a.bps + (g >> 5) * kRecordBytes;
+        c = ld_wire_128(rec + kRecordHeader + lane * 16, pol);
+        s = ld_scale(reinterpret_cast<const float*>(rec) + lane / LPB, pol);
+    } else {
+        c = ld_wire_128(a.codes + slot * a.shard + g * 16, pol);
+        s = ld_scale(a.scales + slot * a.bps + g / LPB, pol);
+    }
     float q[16];
     codes_to_f32x16(c, q);
     Vec8 o;
@@ -260,6 +359,93 @@ __global__ void __launch_bounds__(kThreads) ag_dequant_kernel(const __grid_const
         o.w[i] = pack_bf16x2_rn(__fmul_rn(q[2 * i], s), __fmul_rn(q[2 * i + 1], s));
     const uint64_t byte_off = (k * a.shard + g * 16) * 2;
     for (uint32_t r = 0; r < a.nranks; ++r) st_stream_256(static_cast<char*>(a.out[r]) + byte_off, o);
+}
+
+// Deep-pipelined form of the whole schedule (Section 3.1 pipelines the microshards of a
+// shard through the ring independently; here a microshard is one tile of 512 elements).
+// One warp carries its tile through all N ring steps and the all-gather without waiting
+// for any other tile.  Every hop message still goes through memory as a record: the lane
+// that acts for the sending rank stores its codes (and lanes 0..7 the metadata sector),
+// the warp synchronises, and the NEIGHBOURING lane (lane ^ 1), acting for the receiving
+// rank, loads them back and continues with that 16-element group.  Without a trace the
+// records go to a two-deep staging FIFO that the warp owns and reuses for every step
+// and every tile, the way a ring channel reuses its staging buffers: the FIFO stays in
+// L2 and the hop traffic never reaches HBM.  With a trace every message is kept.
+// The bf16 shard of the next step is prefetched while a step computes.
+constexpr int kPipeThreads = 64;
+#ifndef EQX_PIPE_MINBLOCKS
+#define EQX_PIPE_MINBLOCKS 16
+#endif
+
+template <int LPB>
+__global__ void __launch_bounds__(kPipeThreads, EQX_PIPE_MINBLOCKS) pipelined_kernel(const __grid_constant__ PipeArgs a) {
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint64_t warps = (uint64_t)gridDim.x * (kPipeThreads / 32);
+    const uint64_t warp = (uint64_t)blockIdx.x * (kPipeThreads / 32) + (threadIdx.x >> 5);
+    const uint32_t N = a.nranks;
+    const uint64_t groups = a.shard >> 4;
+    const uint64_t tiles = a.tiles_per_shard * N;
+    char* const fifo = a.records + warp * (2 * kRecordBytes);
+
+    for (uint64_t tile = warp; tile < tiles; tile += warps) {
+        const uint32_t k = (uint32_t)(tile / a.tiles_per_shard);           // shard
+        const uint64_t t = tile - (uint64_t)k * a.tiles_per_shard;
+        const uint64_t g = t * 32 + lane;              // this lane's group at even steps; g ^ 1 at odd steps
+        const bool active = g < groups;                // groups is a multiple of 4: lane pairs are in or out together
+        const uint64_t shard_off = (uint64_t)k * a.shard;
+        char* const trace = a.records + ((uint64_t)k * N * a.tiles_per_shard + t) * kRecordBytes;
+
+        uint32_t rho = k + 1 == N ? 0 : k + 1;         // rank of step 0
+        Vec8 xw = {};
+        if (active) xw = ld_coherent_256(static_cast<const char*>(a.in[rho]) + (shard_off + g * 16) * 2);
+        float v[16];
+        widen_bf16x16(xw, v);
+        uint32_t sub = lane;                           // position inside the tile handled at step j
+        for (uint32_t j = 0;; ++j) {
+            rho = rho + 1 == N ? 0 : rho + 1;
+            if (active && j + 1 < N)                   // the next step's bf16 shard arrives while this step computes
+                xw = ld_coherent_256(static_cast<const char*>(a.in[rho]) + (shard_off + (t * 32 + (sub ^ 1)) * 16) * 2);
+            uint4 codes;
+            float scale;
+            quantize_lane<LPB>(v, codes, scale);
+            char* const rec = a.keep_trace ? trace + (uint64_t)j * a.tiles_per_shard * kRecordBytes
+                                           : fifo + (j & 1u) * kRecordBytes;
+            // the sender's view: position `sub` of the tile
+            {
+                float hdr = __shfl_sync(0xFFFFFFFFu, scale, ((lane * LPB) & 31u) ^ (j & 1u));
+                if (lane >= 32u / LPB) hdr = 0.0f;
+                if (lane < 8 && t * 32 < groups) st_plain_f32(reinterpret_cast<float*>(rec) + lane, hdr);
+                if (active) st_plain_128(rec + kRecordHeader + sub * 16, codes);
+            }
+            __syncwarp();                              // the message is now visible to the neighbouring lane,
+            sub ^= 1;                                  // which acts for the receiving rank on the neighbour's group
+            uint4 c = make_uint4(0, 0, 0, 0);
+            float s = 0.0f;
+            if (active) {
+                c = ld_coherent_128(rec + kRecordHeader + sub * 16);
+                s = ld_coherent_f32(reinterpret_cast<const float*>(rec) + sub / LPB);
+            }
+            float q[16];
+            codes_to_f32x16(c, q);
+            if (j + 1 == N) {                          // all-gather: dequantize to bf16, one store per rank
+                Vec8 o;
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    o.w[i] = pack_bf16x2_rn(__fmul_rn(q[2 * i], s), __fmul_rn(q[2 * i + 1], s));
+                if (active) {
+                    const uint64_t byte_off = (shard_off + (t * 32 + sub) * 16) * 2;
+                    for (uint32_t r = 0; r < N; ++r) st_stream_256(static_cast<char*>(a.out[r]) + byte_off, o);
+                }
+                break;
+            }
+            widen_bf16x16(xw, v);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] = __fmaf_rn(q[i], s, v[i]);
+            // FIFO entry (j & 1) is overwritten at step j+2, after the __syncwarp of step j+1: every
+            // lane's load above has returned by then, because its value feeds the quantization of step j+1
+        }
+        __syncwarp();                                  // the next tile reuses the FIFO
+    }
 }
 
 // Unquantized comparator hop: send = bf16_rne(f32(recv) + f32(local)).

@@ -41,10 +41,13 @@ def to_dev_bf16(words_u16):
     return torch.from_numpy(np.ascontiguousarray(words_u16).view(np.int16)).cuda().view(torch.bfloat16)
 
 
-def run_sim(x_dev, block, keep_trace=False, in_place=False):
-    """x_dev: bf16 CUDA tensor [N, count].  Returns (out [N, count] bf16, workspace Guarded)."""
+def run_sim(x_dev, block, keep_trace=False, in_place=False, variant="steps"):
+    """x_dev: bf16 CUDA tensor [N, count].  Returns (out [N, count] bf16, workspace Guarded).
+    variant: "steps" = equarx_allreduce_sim, "pipelined" = equarx_allreduce_sim_pipelined."""
     n_ranks, count = x_dev.shape
-    wb = eq.allreduce_sim_workspace_bytes(n_ranks, count, block, keep_trace)
+    size_fn = {"steps": eq.allreduce_sim_workspace_bytes,
+               "pipelined": eq.allreduce_sim_pipelined_workspace_bytes}[variant]
+    wb = size_fn(n_ranks, count, block, keep_trace)
     assert wb > 0
     ws = Guarded(wb)
     if in_place:
@@ -55,7 +58,8 @@ def run_sim(x_dev, block, keep_trace=False, in_place=False):
     else:
         ins = [x_dev[r] for r in range(n_ranks)]
         outs = [Guarded(2 * count) for _ in range(n_ranks)]
-    eq.allreduce_sim(ins, outs, n_ranks, count, block, ws, wb, keep_trace, stream_handle())
+    fn = {"steps": eq.allreduce_sim, "pipelined": eq.allreduce_sim_pipelined}[variant]
+    fn(ins, outs, n_ranks, count, block, ws, wb, keep_trace, stream_handle())
     torch.cuda.synchronize()
     ws.check()
     for o in outs:

@@ -43,16 +43,37 @@ def test_status_strings():
 
 
 def test_workspace_bytes():
-    # N=4, n=65536, B=256: shard 16384, 64 blocks per shard
-    assert eq.allreduce_sim_workspace_bytes(4, 65536, 256, False) == 8 * 64 * 4 + 8 * 16384
-    assert eq.allreduce_sim_workspace_bytes(4, 65536, 256, True) == 16 * 64 * 4 + 16 * 16384
-    # scales region is padded to 256 bytes: N=1, one block
-    assert eq.allreduce_sim_workspace_bytes(1, 64, 64, False) == 256 + 2 * 64
+    # N=4, n=65536: shard 16384 = 32 tiles of 512 elements, 544 bytes per record
+    assert eq.allreduce_sim_workspace_bytes(4, 65536, 256, False) == 8 * 32 * 544
+    assert eq.allreduce_sim_workspace_bytes(4, 65536, 256, True) == 16 * 32 * 544
+    # a shard smaller than a tile still takes one record per slot
+    assert eq.allreduce_sim_workspace_bytes(1, 64, 64, False) == 2 * 544
+    assert eq.allreduce_sim_workspace_bytes(3, 3 * 5 * 128, 128, True) == 9 * 2 * 544     # 640 elements: 2 tiles
     assert eq.allreduce_sim_workspace_bytes(3, 65536, 256, False) == 0      # not divisible
     assert eq.allreduce_sim_workspace_bytes(4, 65536, 100, False) == 0
     assert eq.allreduce_sim_workspace_bytes(65, 65 * 256, 256, False) == 0
+    assert eq.allreduce_sim_pipelined_workspace_bytes(4, 65536, 256, False) == binding.PIPELINE_FIFO_BYTES
+    assert eq.allreduce_sim_pipelined_workspace_bytes(4, 65536, 256, True) == 16 * 32 * 544
+    assert eq.allreduce_sim_pipelined_workspace_bytes(4, 65536, 99, True) == 0
     assert eq.allreduce_sim_bf16_workspace_bytes(4, 65536) == 4 * 65536
     assert eq.allreduce_sim_bf16_workspace_bytes(4, 65530) == 0
+
+
+def test_trace_views_unpack_records():
+    import numpy as np
+    n, count, block = 2, 2 * 640, 128          # shard 640 = 5 blocks = 2 tiles (the second one ragged)
+    ws = np.zeros(eq.allreduce_sim_workspace_bytes(n, count, block, True), np.uint8)
+    rec = ws.reshape(4, 2, 544)
+    for slot in range(4):
+        for t in range(2):
+            hdr = np.zeros(8, np.float32)
+            hdr[:4] = [slot * 100 + t * 4 + i for i in range(4)]
+            rec[slot, t, :32] = hdr.view(np.uint8)
+            rec[slot, t, 32:] = (np.arange(512) % 100 + slot).astype(np.int8).view(np.uint8)
+    sc, co = eq.trace_views(ws, n, count, block, True)
+    assert sc.shape == (4, 5) and co.shape == (4, 640)
+    assert list(sc[3]) == [300, 301, 302, 303, 304]
+    assert co[2, 0] == 2 and co[2, 511] == 11 % 100 + 2 and co[2, 512] == 2 and co[2, 639] == 127 % 100 + 2
 
 
 def status_of(fn, *args, **kw):

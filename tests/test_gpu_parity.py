@@ -94,19 +94,34 @@ def test_single_block_and_one_tile_edges(gu, block):
         assert np.array_equal(sc.view(torch.float32).cpu().numpy().view(np.uint32), es.view(np.uint32))
 
 
+VARIANTS = ("steps", "pipelined")
+
+
 def _compare_full(gu, x, block, in_place=False):
+    """Both schedules (one launch per ring step; one deep-pipelined launch) against the oracle:
+    the whole trace of messages and the outputs, bit for bit."""
     n_ranks, count = x.shape
     xd = x.cuda()
-    out, ws = gu.run_sim(xd, block, keep_trace=True, in_place=in_place)
     res = oracle.allreduce(wl.as_u16(x), block, trace=True)
-    sc, co = eq.trace_views(ws.u8, n_ranks, count, block, keep_trace=True)
-    assert np.array_equal(co.cpu().numpy().reshape(res["codes"].shape), res["codes"]), "trace codes"
-    assert np.array_equal(sc.cpu().numpy().view(np.uint32).reshape(res["scales"].shape),
-                          res["scales"].view(np.uint32)), "trace scales"
-    gu.assert_same_words(out, res["out"], "outputs")
-    # the ping-pong (no trace) path is what the bench runs: same outputs
-    out2, _ = gu.run_sim(xd, block, keep_trace=False, in_place=in_place)
-    assert torch.equal(out2.view(torch.int16), out.view(torch.int16))
+    last = {}
+    for variant in VARIANTS:
+        out, ws = gu.run_sim(xd, block, keep_trace=True, in_place=in_place, variant=variant)
+        sc, co = eq.trace_views(ws.u8, n_ranks, count, block, keep_trace=True)
+        assert np.array_equal(co.cpu().numpy().reshape(res["codes"].shape), res["codes"]), f"{variant}: trace codes"
+        assert np.array_equal(sc.cpu().numpy().view(np.uint32).reshape(res["scales"].shape),
+                              res["scales"].view(np.uint32)), f"{variant}: trace scales"
+        gu.assert_same_words(out, res["out"], f"{variant}: outputs")
+        # without a trace (what the bench runs): same outputs; the step schedule leaves the last two
+        # events of every shard in its ping-pong workspace
+        out2, ws2 = gu.run_sim(xd, block, keep_trace=False, in_place=in_place, variant=variant)
+        assert torch.equal(out2.view(torch.int16), out.view(torch.int16)), variant
+        if variant == "steps":
+            sc2, co2 = eq.trace_views(ws2.u8, n_ranks, count, block, keep_trace=False)
+            for k in range(n_ranks):
+                for j in range(max(0, n_ranks - 2), n_ranks):
+                    assert np.array_equal(co2[2 * k + (j & 1)].cpu().numpy(), res["codes"][k, j]), (k, j)
+                    assert np.array_equal(sc2[2 * k + (j & 1)].cpu().numpy().view(np.uint32),
+                                          res["scales"][k, j].view(np.uint32)), (k, j)
 
 
 def test_config1_small_normal_full(gu):
@@ -141,12 +156,13 @@ def test_in_place(gu):
     _compare_full(gu, wl.make_inputs(w), 256, in_place=True)
 
 
+@pytest.mark.parametrize("variant", VARIANTS)
 @pytest.mark.parametrize("w", [wl.C2, wl.C3, wl.C5], ids=lambda w: w.name)
-def test_full_size_sampled(gu, w):
+def test_full_size_sampled(gu, w, variant):
     """Full-size configs in the launch configuration the bench times (ping-pong workspace):
     outputs of sampled blocks bit for bit, plus properties that hold at any size."""
     x = wl.make_inputs(w, device="cuda")
-    out, ws = gu.run_sim(x, w.block, keep_trace=False)
+    out, ws = gu.run_sim(x, w.block, keep_trace=False, variant=variant)
     for r in range(1, w.nranks):
         assert torch.equal(out[0].view(torch.int16), out[r].view(torch.int16)), "outputs differ across ranks"
     bps = w.count // w.nranks // w.block
@@ -154,13 +170,14 @@ def test_full_size_sampled(gu, w):
     exp = gu.oracle_out_on_samples(x, picks, w.block)
     got = gu.gather_blocks(out, picks, w.block)
     gu.assert_same_words(got, exp, "sampled outputs")
-    # the last two messages of every rank are still in the workspace: codes within +-127
-    # and, per block, scale 0 or at least one |code| == 127
-    sc, co = eq.trace_views(ws.u8, w.nranks, w.count, w.block, keep_trace=False)
-    assert int(co.min()) >= -127
-    amax = co.view(2 * w.nranks, -1, w.block).abs().amax(dim=2)
-    assert bool(((amax == 127) | (sc == 0)).all())
-    assert bool(((sc != 0) | (amax == 0)).all())
+    if variant == "steps":
+        # the last two messages of every shard are still in the workspace: codes within +-127
+        # and, per block, scale 0 or at least one |code| == 127
+        sc, co = eq.trace_views(ws.u8, w.nranks, w.count, w.block, keep_trace=False)
+        assert int(co.min()) >= -127
+        amax = co.view(2 * w.nranks, -1, w.block).abs().amax(dim=2)
+        assert bool(((amax == 127) | (sc == 0)).all())
+        assert bool(((sc != 0) | (amax == 0)).all())
 
 
 @pytest.mark.parametrize("nranks,count", [(1, 4096), (2, 2 * 4096 + 32), (4, 65536), (7, 7 * 16 * 301), (64, 64 * 4096)])
