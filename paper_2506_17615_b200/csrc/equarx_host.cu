@@ -48,8 +48,6 @@ inline int check_sim_shape(int nranks, size_t count, int block) {
     return EQUARX_OK;
 }
 
-inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
-
 // Programmatic dependent launch is on unless EQUARX_PDL=0 (read once).
 bool use_pdl() {
     static const bool on = [] {
@@ -163,6 +161,7 @@ int equarx_quantize_blocks(const void* x_bf16, size_t count, int block, int8_t* 
         overlap(codes, count, scales, 4 * (count / block)))
         return EQUARX_ERR_ALIAS;
     StepArgs a = {};
+    a.neg_zero = -0.0f;
     a.x[0] = x_bf16;
     a.codes_out = codes;
     a.scales_out = scales;
@@ -186,6 +185,7 @@ int equarx_rs_step_dequant_add_requant(const int8_t* codes_in, const float* scal
         for (int j = 3; j < 5; ++j)
             if (i != j && overlap(bufs[i], lens[i], bufs[j], lens[j])) return EQUARX_ERR_ALIAS;
     StepArgs a = {};
+    a.neg_zero = -0.0f;
     a.x[0] = local_bf16;
     a.codes_in = codes_in;
     a.scales_in = scales_in;
@@ -248,6 +248,7 @@ int equarx_allreduce_sim_range(const void* const* in_bf16, void* const* out_bf16
     };
 
     StepArgs a = {};
+    a.neg_zero = -0.0f;
     a.codes_in = records;
     a.codes_out = records;
     a.shard = shard;
@@ -297,6 +298,7 @@ int equarx_allreduce_sim_pipelined(const void* const* in_bf16, void* const* out_
     const uint32_t N = uint32_t(nranks);
     const size_t shard = count / N;
     PipeArgs a = {};
+    a.neg_zero = -0.0f;
     for (uint32_t r = 0; r < N; ++r) {
         a.in[r] = in_bf16[r];
         a.out[r] = out_bf16[r];

@@ -11,9 +11,10 @@
 // Every floating-point step that decides a bit of the result uses an explicit
 // round-to-nearest intrinsic, so the compiler cannot contract or reorder it:
 //   scale = __fdiv_rn(amax, 127), inv = __fdiv_rn(127, amax)
-//   code  = rne(__fmul_rn(v, inv))    (the add of 1.5*2^23 rounds to the integer grid)
-//   hop   = __fmaf_rn((float)code, scale, local)
-//   final = cvt.rn.bf16(__fmul_rn((float)code, scale))
+//   code  = rne(mul.rn(v, inv))       (the add.rn of 1.5*2^23 rounds to the integer grid)
+//   hop   = fma.rn((float)code, scale, local)
+//   final = cvt.rn.bf16(mul.rn((float)code, scale))
+// (mul/add/fma are the packed .f32x2 forms of sm_100: two IEEE results per instruction.)
 #pragma once
 #include <cstdint>
 #include <cuda_runtime.h>
@@ -128,6 +129,31 @@ __device__ __forceinline__ void pdl_wait_prior_grid() {
 }
 
 // ---------------------------------------------------------------- arithmetic
+// sm_100 packed fp32: one instruction, two independent IEEE round-to-nearest results.
+// The path is bound by instruction issue as much as by memory, so halving the count of
+// the multiplies and adds matters; each half rounds exactly like the scalar intrinsic.
+__device__ __forceinline__ void fma2_rn(float& d0, float& d1, float a0, float a1, float b, float c0, float c1) {
+    asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\tmov.b64 rc, {%5, %6};\n\t"
+        "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d0), "=f"(d1)
+        : "f"(a0), "f"(a1), "f"(b), "f"(c0), "f"(c1));
+}
+__device__ __forceinline__ void mul2_rn(float& d0, float& d1, float a0, float a1, float b) {
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\t"
+        "mul.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d0), "=f"(d1)
+        : "f"(a0), "f"(a1), "f"(b));
+}
+__device__ __forceinline__ void add2_rn(float& d0, float& d1, float a0, float a1, float b) {
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\t"
+        "add.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d0), "=f"(d1)
+        : "f"(a0), "f"(a1), "f"(b));
+}
+
 // bf16 -> fp32 is exact: the bf16 word is the upper half of the fp32 word.
 __device__ __forceinline__ void widen_bf16x16(const Vec8& x, float (&v)[16]) {
 #pragma unroll
@@ -144,11 +170,36 @@ __device__ __forceinline__ void codes_to_f32x16(const uint4& c, float (&q)[16]) 
     const uint32_t w[4] = {c.x ^ 0x80808080u, c.y ^ 0x80808080u, c.z ^ 0x80808080u, c.w ^ 0x80808080u};
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-        q[4 * j + 0] = __fsub_rn(__uint_as_float(__byte_perm(w[j], 0x4B000000u, 0x7540)), 8388736.0f);
-        q[4 * j + 1] = __fsub_rn(__uint_as_float(__byte_perm(w[j], 0x4B000000u, 0x7541)), 8388736.0f);
-        q[4 * j + 2] = __fsub_rn(__uint_as_float(__byte_perm(w[j], 0x4B000000u, 0x7542)), 8388736.0f);
-        q[4 * j + 3] = __fsub_rn(__uint_as_float(__byte_perm(w[j], 0x4B000000u, 0x7543)), 8388736.0f);
+        const float u0 = __uint_as_float(__byte_perm(w[j], 0x4B000000u, 0x7540));
+        const float u1 = __uint_as_float(__byte_perm(w[j], 0x4B000000u, 0x7541));
+        const float u2 = __uint_as_float(__byte_perm(w[j], 0x4B000000u, 0x7542));
+        const float u3 = __uint_as_float(__byte_perm(w[j], 0x4B000000u, 0x7543));
+        add2_rn(q[4 * j + 0], q[4 * j + 1], u0, u1, -8388736.0f);
+        add2_rn(q[4 * j + 2], q[4 * j + 3], u2, u3, -8388736.0f);
     }
+}
+
+// v[i] = fma((float)code[i], scale, v[i]): the hop's dequantize-and-add, one rounding.
+__device__ __forceinline__ void dequant_add_x16(const uint4& c, float scale, float (&v)[16]) {
+    float q[16];
+    codes_to_f32x16(c, q);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) fma2_rn(v[2 * i], v[2 * i + 1], q[2 * i], q[2 * i + 1], scale, v[2 * i], v[2 * i + 1]);
+}
+
+// bf16x2 words of (float)code[i] * scale, rounded to nearest even: the all-gather dequantize.
+__device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi);
+__device__ __forceinline__ Vec8 dequant_to_bf16x16(const uint4& c, float scale) {
+    float q[16];
+    codes_to_f32x16(c, q);
+    Vec8 o;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        float lo, hi;
+        mul2_rn(lo, hi, q[2 * i], q[2 * i + 1], scale);
+        o.w[i] = pack_bf16x2_rn(lo, hi);
+    }
+    return o;
 }
 
 template <int LPB>
@@ -173,7 +224,7 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 // lanes 127/amax; the operands are selected, the instruction stream is the same) and
 // the pair of lanes exchanges the quotients with two shuffles.
 template <int LPB>
-__device__ __forceinline__ void quantize_lane(const float (&v)[16], uint4& codes, float& scale) {
+__device__ __forceinline__ void quantize_lane(const float (&v)[16], uint4& codes, float& scale, float neg_zero) {
     float m = max3(fabsf(v[0]), fabsf(v[1]), fabsf(v[2]));
     float m1 = max3(fabsf(v[3]), fabsf(v[4]), fabsf(v[5]));
     float m2 = max3(fabsf(v[6]), fabsf(v[7]), fabsf(v[8]));
@@ -189,8 +240,19 @@ __device__ __forceinline__ void quantize_lane(const float (&v)[16], uint4& codes
     const float inv = __shfl_sync(0xFFFFFFFFu, keep, (threadIdx.x & 30u) | 1u);
     uint32_t b[16];
 #pragma unroll
-    for (int i = 0; i < 16; ++i)
-        b[i] = __float_as_uint(__fadd_rn(__fmul_rn(v[i], inv), 12582912.0f));
+    for (int i = 0; i < 8; ++i) {
+        // The product must be rounded to fp32 BEFORE the add of 1.5 * 2^23 (two roundings, as in
+        // rintf(v * inv)).  ptxas contracts a packed mul.rn.f32x2 (or a packed fma with a literal
+        // zero addend) feeding a packed add.rn.f32x2 into one fused multiply-add (seen on ties:
+        // 63.5 -> 63 instead of 64).  So the product is formed by a packed fma whose addend is
+        // -0.0 passed in as a kernel argument: it leaves every product unchanged, the compiler
+        // cannot fold it away, and an fma cannot be merged with the following add.
+        float t0, t1, r0, r1;
+        fma2_rn(t0, t1, v[2 * i], v[2 * i + 1], inv, neg_zero, neg_zero);
+        add2_rn(r0, r1, t0, t1, 12582912.0f);
+        b[2 * i] = __float_as_uint(r0);
+        b[2 * i + 1] = __float_as_uint(r1);
+    }
     uint32_t o[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
@@ -240,6 +302,7 @@ struct StepArgs {
     float* scales_out;
     uint64_t shard;                  // elements per message
     uint64_t bps;                    // SPLIT: blocks per message; RECORDS: bytes per slot
+    float neg_zero;                  // -0.0f, opaque to the compiler (see quantize_lane)
 };
 
 struct GatherArgs {
@@ -260,6 +323,7 @@ struct PipeArgs {
     uint64_t tiles_per_shard;        // 512-element tiles per shard (the last one may be ragged)
     uint32_t nranks;
     uint32_t keep_trace;
+    float neg_zero;                  // -0.0f, opaque to the compiler (see quantize_lane)
 };
 
 struct Bf16StepArgs {
@@ -310,15 +374,12 @@ __global__ void __launch_bounds__(kThreads) rs_step_kernel(const __grid_constant
                 s = ld_scale(a.scales_in + slot * a.bps + g / LPB, pol);
             }
         }
-        float q[16];
-        codes_to_f32x16(c, q);
-#pragma unroll
-        for (int i = 0; i < 16; ++i) v[i] = __fmaf_rn(q[i], s, v[i]);
+        dequant_add_x16(c, s, v);
     }
 
     uint4 codes;
     float scale;
-    quantize_lane<LPB>(v, codes, scale);
+    quantize_lane<LPB>(v, codes, scale, a.neg_zero);
     const uint64_t slot = a.out_slot[r];
     if (RECORDS) {
         char* rec = reinterpret_cast<char*>(a.codes_out) + slot * a.bps + (g >> 5) * kRecordBytes;
@@ -351,12 +412,7 @@ __global__ void __launch_bounds__(kThreads) ag_dequant_kernel(const __grid_const
         c = ld_wire_128(a.codes + slot * a.shard + g * 16, pol);
         s = ld_scale(a.scales + slot * a.bps + g / LPB, pol);
     }
-    float q[16];
-    codes_to_f32x16(c, q);
-    Vec8 o;
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-        o.w[i] = pack_bf16x2_rn(__fmul_rn(q[2 * i], s), __fmul_rn(q[2 * i + 1], s));
+    const Vec8 o = dequant_to_bf16x16(c, s);
     const uint64_t byte_off = (k * a.shard + g * 16) * 2;
     for (uint32_t r = 0; r < a.nranks; ++r) st_stream_256(static_cast<char*>(a.out[r]) + byte_off, o);
 }
@@ -407,7 +463,7 @@ __global__ void __launch_bounds__(kPipeThreads, EQX_PIPE_MINBLOCKS) pipelined_ke
                 xw = ld_coherent_256(static_cast<const char*>(a.in[rho]) + (shard_off + (t * 32 + (sub ^ 1)) * 16) * 2);
             uint4 codes;
             float scale;
-            quantize_lane<LPB>(v, codes, scale);
+            quantize_lane<LPB>(v, codes, scale, a.neg_zero);
             char* const rec = a.keep_trace ? trace + (uint64_t)j * a.tiles_per_shard * kRecordBytes
                                            : fifo + (j & 1u) * kRecordBytes;
             // the sender's view: position `sub` of the tile
@@ -425,13 +481,8 @@ __global__ void __launch_bounds__(kPipeThreads, EQX_PIPE_MINBLOCKS) pipelined_ke
                 c = ld_coherent_128(rec + kRecordHeader + sub * 16);
                 s = ld_coherent_f32(reinterpret_cast<const float*>(rec) + sub / LPB);
             }
-            float q[16];
-            codes_to_f32x16(c, q);
             if (j + 1 == N) {                          // all-gather: dequantize to bf16, one store per rank
-                Vec8 o;
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    o.w[i] = pack_bf16x2_rn(__fmul_rn(q[2 * i], s), __fmul_rn(q[2 * i + 1], s));
+                const Vec8 o = dequant_to_bf16x16(c, s);
                 if (active) {
                     const uint64_t byte_off = (shard_off + (t * 32 + sub) * 16) * 2;
                     for (uint32_t r = 0; r < N; ++r) st_stream_256(static_cast<char*>(a.out[r]) + byte_off, o);
@@ -439,8 +490,7 @@ __global__ void __launch_bounds__(kPipeThreads, EQX_PIPE_MINBLOCKS) pipelined_ke
                 break;
             }
             widen_bf16x16(xw, v);
-#pragma unroll
-            for (int i = 0; i < 16; ++i) v[i] = __fmaf_rn(q[i], s, v[i]);
+            dequant_add_x16(c, s, v);
             // FIFO entry (j & 1) is overwritten at step j+2, after the __syncwarp of step j+1: every
             // lane's load above has returned by then, because its value feeds the quantization of step j+1
         }
