@@ -316,8 +316,7 @@ int equarx_allreduce_sim_pipelined(const void* const* in_bf16, void* const* out_
         case 256: kernel = reinterpret_cast<const void*>(pipelined_kernel<16>); break;
         default: kernel = reinterpret_cast<const void*>(pipelined_kernel<32>); break;
     }
-    // persistent grid: a whole number of CTAs per SM, chosen so that the warp tiles split
-    // into full rounds as evenly as possible
+    // persistent grid: a whole number of CTAs per SM
     int dev = 0, sms = 0, occ = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -327,15 +326,16 @@ int equarx_allreduce_sim_pipelined(const void* const* in_bf16, void* const* out_
         (void)cudaGetLastError();
         return EQUARX_ERR_CUDA;
     }
+    // The kernel is bound by the latency of the per-tile chain, so a round (every warp carries one
+    // tile through the ring) costs about the same whatever the number of resident warps: take the
+    // CTA count per SM that needs the fewest rounds and, among those, the smallest one.
     const uint64_t tiles = a.tiles_per_shard * N, wpc = kPipeThreads / 32;
-    uint64_t best_ctas = 0;
-    double best_eff = -1.0;
-    for (int c = occ; c >= (occ + 1) / 2; --c) {
+    uint64_t best_ctas = 0, best_rounds = ~uint64_t(0);
+    for (int c = 1; c <= occ; ++c) {
         const uint64_t ctas = uint64_t(sms) * c, w = ctas * wpc;
         const uint64_t rounds = (tiles + w - 1) / w;
-        const double eff = double(tiles) / double(rounds * w);
-        if (eff > best_eff + 1e-9) {
-            best_eff = eff;
+        if (rounds < best_rounds) {
+            best_rounds = rounds;
             best_ctas = ctas;
         }
     }

@@ -1,0 +1,112 @@
+"""Message-size sweep of the simulated quantized AllReduce (config 4 of the benchmark definition).
+
+    python -m paper_2506_17615_b200.sweep [--out sweep.jsonl] [--quick]
+
+For every point (N in {4, 8, 16}, block in {128, 256, 512}, uniform(-1,1) and N(0,1), per-rank
+messages from 16 KB to 256 MB in powers of two) it times, with CUDA events and inputs resident in
+device memory, the pipelined schedule, the launch-per-step schedule and the unquantized bf16 ring,
+and prints one JSON line per point: GB/s of bf16 input reduced and the fraction of the HBM
+roofline (algorithmic bytes n*N*(6+8/B) over the measured copy bandwidth).  Inputs rotate over
+several resident sets so that consecutive iterations do not find their inputs in L2.
+"""
+import argparse
+import json
+import os
+import sys
+
+import torch
+
+import paper_2506_17615_b200 as eq
+from paper_2506_17615_b200 import workloads as wl
+
+
+def hbm_peak_gbs():
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    try:
+        with open(os.path.join(root, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def time_ms(fn, iters, warmup=3):
+    for i in range(warmup):
+        fn(i)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for i in range(iters):
+        fn(i)
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / iters
+
+
+def run_point(n_ranks, nbytes, block, dist, peak):
+    w = wl.sweep_point(n_ranks, nbytes, block, dist)
+    count = w.count
+    if count % (n_ranks * block):
+        return None
+    in_bytes = 2 * count * n_ranks
+    sets = 1 if in_bytes > 1_000_000_000 else min(16, max(2, -(-378_000_000 // (2 * in_bytes))))
+    base = wl.make_inputs(w, device="cuda")
+    ins, outs = [], []
+    for s in range(sets):
+        x = base if s == 0 else base.roll(s * 4096, dims=1).contiguous()    # same values, other addresses
+        ins.append([x[r] for r in range(n_ranks)])
+        o = torch.empty_like(x)
+        outs.append([o[r] for r in range(n_ranks)])
+    stream = torch.cuda.current_stream().cuda_stream
+    wb = eq.allreduce_sim_workspace_bytes(n_ranks, count, block, False)
+    ws = torch.empty(wb, dtype=torch.uint8, device="cuda")
+    wbp = eq.allreduce_sim_pipelined_workspace_bytes(n_ranks, count, block, False)
+    wsp = torch.empty(wbp, dtype=torch.uint8, device="cuda")
+    wb16 = eq.allreduce_sim_bf16_workspace_bytes(n_ranks, count)
+    ws16 = torch.empty(wb16, dtype=torch.uint8, device="cuda")
+    iters = max(5, min(200, int(2e9 // max(in_bytes, 1))))
+    t_pipe = time_ms(lambda i: eq.allreduce_sim_pipelined(ins[i % sets], outs[i % sets], n_ranks, count, block,
+                                                          wsp, wbp, False, stream), iters)
+    t_steps = time_ms(lambda i: eq.allreduce_sim(ins[i % sets], outs[i % sets], n_ranks, count, block,
+                                                 ws, wb, False, stream), iters)
+    t_bf16 = time_ms(lambda i: eq.allreduce_sim_bf16(ins[i % sets], outs[i % sets], n_ranks, count,
+                                                     ws16, wb16, stream), iters)
+    alg = count * n_ranks * (6 + 8 / block)
+    alg16 = count * (8 * n_ranks - 4)
+    gbs = lambda nbytes_, ms: nbytes_ / (ms * 1e-3) / 1e9
+    return {"nranks": n_ranks, "bytes_per_rank": nbytes, "block": block, "dist": dist, "iters": iters, "sets": sets,
+            "pipelined": {"ms": t_pipe, "gbs_in": gbs(in_bytes, t_pipe), "frac": gbs(alg, t_pipe) / peak},
+            "by_steps": {"ms": t_steps, "gbs_in": gbs(in_bytes, t_steps), "frac": gbs(alg, t_steps) / peak},
+            "bf16_sim": {"ms": t_bf16, "gbs_in": gbs(in_bytes, t_bf16), "frac": gbs(alg16, t_bf16) / peak}}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--out", default=None)
+    ap.add_argument("--quick", action="store_true", help="block 256 and N(0,1) only")
+    args = ap.parse_args()
+    if not torch.cuda.is_available():
+        raise SystemExit("the sweep needs a CUDA device")
+    peak, src = hbm_peak_gbs()
+    out = open(args.out, "w") if args.out else None
+    blocks = (256,) if args.quick else (128, 256, 512)
+    dists = ("normal",) if args.quick else ("uniform", "normal")
+    for n_ranks in (4, 8, 16):
+        for block in blocks:
+            for dist in dists:
+                for p in range(14, 29):
+                    rec = run_point(n_ranks, 1 << p, block, dist, peak)
+                    if rec is None:
+                        continue
+                    rec["peak_gbs"], rec["peak_source"] = peak, src
+                    line = json.dumps(rec)
+                    print(line, flush=True)
+                    if out:
+                        out.write(line + "\n")
+                        out.flush()
+                    torch.cuda.empty_cache()
+    if out:
+        out.close()
+
+
+if __name__ == "__main__":
+    sys.exit(main())
