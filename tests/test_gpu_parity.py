@@ -227,3 +227,40 @@ def test_launch_ranges_compose_to_the_whole_schedule(gu):
         assert torch.equal(outs[r].view(torch.int16), ref[r].view(torch.int16))
     with pytest.raises(eq.EquarxError):
         eq.allreduce_sim_range(ins, outs, 5, w.count, 256, ws, wb, False, 2, 6, gu.stream_handle())
+
+
+SWEEP_SMALL = [(n, b, d, s) for n in (4, 8, 16) for b in (128, 256, 512) for d in ("uniform", "normal")
+               for s in (1 << 14, 1 << 17, 1 << 20)]
+
+
+@pytest.mark.parametrize("nranks,block,dist,nbytes", SWEEP_SMALL)
+def test_sweep_points_small_full_compare(gu, nranks, block, dist, nbytes):
+    """Message-size sweep, 16 KB .. 1 MB per rank: every output word of both schedules."""
+    w = wl.sweep_point(nranks, nbytes, block, dist)
+    x = wl.make_inputs(w)
+    exp = oracle.allreduce(wl.as_u16(x), block)["out"]
+    xd = x.cuda()
+    for variant in VARIANTS:
+        out, _ = gu.run_sim(xd, block, variant=variant)
+        gu.assert_same_words(out, exp, f"{variant} {w.name}")
+
+
+SWEEP_LARGE = [(n, b, "uniform" if (n + b) % 3 else "normal", s) for n in (4, 8, 16) for b in (128, 256, 512)
+               for s in (1 << 24, 1 << 26, 1 << 28)]
+
+
+@pytest.mark.parametrize("nranks,block,dist,nbytes", SWEEP_LARGE)
+def test_sweep_points_large_sampled(gu, nranks, block, dist, nbytes):
+    """16 MB, 64 MB and 256 MB per rank, one distribution per (N, block): sampled blocks bit for bit,
+    all ranks' outputs identical."""
+    w = wl.sweep_point(nranks, nbytes, block, dist)
+    x = wl.make_inputs(w, device="cuda")
+    picks = gu.sample_blocks(nranks, w.count // nranks // block, 12, seed=nbytes % 1000 + nranks)
+    exp = gu.oracle_out_on_samples(x, picks, block)
+    for variant in VARIANTS:
+        out, _ = gu.run_sim(x, block, variant=variant)
+        for r in range(1, nranks):
+            assert torch.equal(out[0].view(torch.int16), out[r].view(torch.int16))
+        gu.assert_same_words(gu.gather_blocks(out, picks, block), exp, f"{variant} {w.name}")
+        del out
+    torch.cuda.empty_cache()
