@@ -15,5 +15,6 @@ from .binding import (  # noqa: F401
     ag_dequant,
     allreduce,
     allreduce_bf16,
+    allreduce_variant,
     error_bound,
 )

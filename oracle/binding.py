@@ -50,9 +50,10 @@ def _load():
         lib.equarx_oracle_ag_dequant.argtypes = [vp, vp, sz, ci, vp]
         lib.equarx_oracle_allreduce.argtypes = [vp, vp, ci, sz, ci, vp, vp, vp]
         lib.equarx_oracle_allreduce_bf16.argtypes = [vp, vp, ci, sz]
+        lib.equarx_oracle_allreduce_variant.argtypes = [vp, vp, ci, sz, ci, ci, ci, ci, vp, vp]
         lib.equarx_oracle_error_bound.argtypes = [vp, vp, ci, sz, ci, vp]
         for name in ("quantize_blocks", "rs_step", "ag_dequant", "allreduce",
-                     "allreduce_bf16", "error_bound"):
+                     "allreduce_bf16", "error_bound", "allreduce_variant"):
             getattr(lib, "equarx_oracle_" + name).restype = ci
         _lib = lib
     return _lib
@@ -143,6 +144,29 @@ def allreduce(inputs_bf16, block, trace=False, exact=False):
         _ptr_array(rows_in), _ptr_array(rows_out), n_ranks, count, block,
         _p(ts) if trace else None, _p(tc) if trace else None, _p(ex) if exact else None),
         "allreduce")
+    return res
+
+
+def allreduce_variant(inputs_bf16, block, semi_loop=False, quant_rs=True, quant_ag=True, trace=False):
+    """The flavours of Sections 3.3 / 3.4: full-loop or semi-loop ring, with the reduce-scatter
+    hops and/or the all-gather quantized.  Returns a dict like allreduce()."""
+    x = _arr(inputs_bf16, np.uint16)
+    n_ranks, count = x.shape
+    if block < 1:
+        raise OracleError(3, "allreduce_variant")
+    if count == 0 or count % (n_ranks * block):
+        raise OracleError(4, "allreduce_variant")
+    out = np.empty_like(x)
+    res = {"out": out}
+    ts = tc = None
+    if trace:
+        ts = np.empty((n_ranks, n_ranks, count // n_ranks // block), np.float32)
+        tc = np.empty((n_ranks, n_ranks, count // n_ranks), np.int8)
+        res["scales"], res["codes"] = ts, tc
+    _check(_load().equarx_oracle_allreduce_variant(
+        _ptr_array([x[r] for r in range(n_ranks)]), _ptr_array([out[r] for r in range(n_ranks)]),
+        n_ranks, count, block, int(semi_loop), int(quant_rs), int(quant_ag),
+        _p(ts) if trace else None, _p(tc) if trace else None), "allreduce_variant")
     return res
 
 

@@ -335,6 +335,145 @@ int equarx_oracle_allreduce_bf16(const uint16_t *const *in, uint16_t *const *out
 }
 
 /*
+ * The other flavours of Section 3.3 / 3.4, written per shard as the adder chains
+ * of Fig. 4 and Fig. 5 (blocks are independent, so the order of shards and
+ * blocks is immaterial):
+ *
+ *   semi_loop = 0: full-loop chain  k+1 -> k+2 -> ... -> k-1 -> k      (N-1 hops)
+ *   semi_loop = 1: two half chains that meet at the owner k (N even):
+ *                  A: k+N/2 -> k+N/2-1 -> ... -> k+1 -> k              (N/2 hops)
+ *                  B: k+N/2+1 -> k+N/2+2 -> ... -> k-1 -> k            (N/2-1 hops)
+ *                  (on 4 devices: 2 -> 1 -> 0 and 3 -> 0, the example of Section 3.3);
+ *                  B's partial reaches the owner one iteration before A's, so the
+ *                  owner adds B's first, then A's.
+ *   quant_rs     : hop messages are quantized (else bf16: the add is rounded to
+ *                  bf16 at every hop, as in the BF16 baseline);
+ *   quant_ag     : the reduced shard goes through one more quantize/dequantize
+ *                  pair (else the owner's result is rounded to bf16 and
+ *                  forwarded as is).
+ * With quant_rs the partial sum stays fp32 from the fused add to the next
+ * quantization, also on the semi-loop owner between its two receives.  Without
+ * quant_rs the reduce-scatter result is a bf16 tensor, and that is what a
+ * quantized all-gather then quantizes.
+ *
+ * Trace (optional, same shapes as equarx_oracle_allreduce): event j of shard k is
+ *   full loop : j = 0..N-2 the hops in chain order, j = N-1 the all-gather message;
+ *   semi loop : j = 0..N/2-1 chain A's hops, j = N/2..N-2 chain B's hops, j = N-1
+ *               the all-gather message.
+ * Events that are not quantized in the chosen flavour are left zero.
+ */
+static void hop_receive(int quant, const float *v_sent, int block, const float *addend,
+                        int addend_is_bf16_exact, float *v_out, int8_t *codes, float *scale)
+{
+    /* sender side: message of v_sent; receiver side: v_out = message (+) addend */
+    (void)addend_is_bf16_exact;
+    if (quant) {
+        quantize_one_block(v_sent, block, codes, scale);
+        for (int i = 0; i < block; ++i) v_out[i] = fmaf((float)codes[i], *scale, addend[i]);
+    } else {
+        for (int i = 0; i < block; ++i) {
+            float msg = bf16_to_f32(f32_to_bf16_rne(v_sent[i]));      /* the bf16 message */
+            v_out[i] = bf16_to_f32(f32_to_bf16_rne(msg + addend[i])); /* add, rounded to bf16 */
+        }
+    }
+}
+
+int equarx_oracle_allreduce_variant(const uint16_t *const *in, uint16_t *const *out,
+                                    int nranks, size_t count, int block,
+                                    int semi_loop, int quant_rs, int quant_ag,
+                                    float *trace_scales, int8_t *trace_codes)
+{
+    if (!in || !out) return ORACLE_ERR_NULL;
+    int st = check_sim_args(nranks, count, block);
+    if (st) return st;
+    if (semi_loop && (nranks % 2 != 0)) return ORACLE_ERR_NRANKS;
+    const size_t N = (size_t)nranks;
+    const size_t shard = count / N;
+    const size_t bps = shard / (size_t)block;
+    for (size_t r = 0; r < N; ++r) {
+        if (!in[r] || !out[r]) return ORACLE_ERR_NULL;
+        for (size_t e = 0; e < count; ++e)
+            if (!bf16_is_finite(in[r][e])) return ORACLE_ERR_NONFINITE;
+    }
+    if (trace_scales) memset(trace_scales, 0, N * N * bps * sizeof(float));
+    if (trace_codes) memset(trace_codes, 0, N * N * shard);
+
+    float *v = (float *)malloc(4 * (size_t)block * sizeof(float));
+    int8_t *codes = (int8_t *)malloc((size_t)block);
+    if (!v || !codes) { free(v); free(codes); return ORACLE_ERR_ALLOC; }
+    float *x = v + block, *acc = v + 2 * (size_t)block, *w = v + 3 * (size_t)block;
+
+    for (size_t k = 0; k < N; ++k) {
+        for (size_t b = 0; b < bps; ++b) {
+            const size_t base = k * shard + b * (size_t)block;
+            size_t event = 0;
+            float scale;
+#define LOAD(dst, rank) for (int i = 0; i < block; ++i) (dst)[i] = bf16_to_f32(in[(rank) % N][base + (size_t)i])
+#define RECORD(quantized) do { if (quantized) { \
+                if (trace_scales) trace_scales[(k * N + event) * bps + b] = scale; \
+                if (trace_codes) memcpy(trace_codes + (k * N + event) * shard + b * (size_t)block, codes, (size_t)block); } \
+                ++event; } while (0)
+            if (!semi_loop) {
+                LOAD(v, k + 1);
+                for (size_t j = 1; j < N; ++j) {           /* hop into rank k+1+j */
+                    LOAD(x, k + 1 + j);
+                    hop_receive(quant_rs, v, block, x, 1, w, codes, &scale);
+                    memcpy(v, w, (size_t)block * sizeof(float));
+                    RECORD(quant_rs);
+                }
+                memcpy(acc, v, (size_t)block * sizeof(float));
+            } else {
+                const size_t h = N / 2;
+                /* chain B first: it reaches the owner one iteration earlier */
+                LOAD(acc, k);
+                size_t event_b = h;                        /* B's events follow A's in the trace */
+                if (h >= 2) {
+                    LOAD(v, k + h + 1);
+                    for (size_t j = 1; j < h; ++j) {       /* B has h-1 ranks: k+h+1 .. k+N-1 */
+                        const int last = (j == h - 1);
+                        if (!last) LOAD(x, k + h + 1 + j);
+                        event = event_b++;
+                        hop_receive(quant_rs, v, block, last ? acc : x, 1, w, codes, &scale);
+                        RECORD(quant_rs);
+                        memcpy(last ? acc : v, w, (size_t)block * sizeof(float));
+                    }
+                }
+                /* chain A: k+h -> k+h-1 -> ... -> k+1 -> owner */
+                LOAD(v, k + h);
+                event = 0;
+                for (size_t j = 1; j <= h; ++j) {
+                    const int last = (j == h);
+                    if (!last) LOAD(x, k + h - j);
+                    hop_receive(quant_rs, v, block, last ? acc : x, 1, w, codes, &scale);
+                    RECORD(quant_rs);
+                    memcpy(last ? acc : v, w, (size_t)block * sizeof(float));
+                }
+            }
+            /* acc is the owner's reduced block: fp32 if the hops were quantized, else a bf16 value */
+            event = N - 1;
+            if (quant_ag) {
+                quantize_one_block(acc, block, codes, &scale);
+                RECORD(1);
+                for (int i = 0; i < block; ++i) {
+                    uint16_t h16 = f32_to_bf16_rne((float)codes[i] * scale);
+                    for (size_t r = 0; r < N; ++r) out[r][base + (size_t)i] = h16;
+                }
+            } else {
+                for (int i = 0; i < block; ++i) {
+                    uint16_t h16 = f32_to_bf16_rne(acc[i]);
+                    for (size_t r = 0; r < N; ++r) out[r][base + (size_t)i] = h16;
+                }
+            }
+#undef LOAD
+#undef RECORD
+        }
+    }
+    free(v);
+    free(codes);
+    return ORACLE_OK;
+}
+
+/*
  * A-posteriori error bound of the quantized AllReduce against the exact sum,
  * from the scales of the trace: every quantize event j of a block moves a
  * value by at most half a quantization step scale_j (plus the fp32 rounding
