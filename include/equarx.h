@@ -60,8 +60,9 @@ enum equarx_status {
     EQUARX_ERR_WORKSPACE = 6,  /* workspace_bytes smaller than *_workspace_bytes()       */
     EQUARX_ERR_ALIAS = 7,      /* buffers overlap in a way the call does not allow       */
     EQUARX_ERR_CUDA = 8,       /* a launch failed; see equarx_last_cuda_error()          */
-    EQUARX_ERR_STATIC_LIMIT = 9 /* problem too large for the built-in workspace of
+    EQUARX_ERR_STATIC_LIMIT = 9, /* problem too large for the built-in workspace of
                                   equarx_allreduce_sim_static                            */
+    EQUARX_ERR_FLAVOUR = 10    /* flavour is not a combination of EQUARX_FLAVOUR_* bits  */
 };
 
 /*
@@ -179,6 +180,43 @@ int equarx_allreduce_sim_pipelined(const void *const *in_bf16, void *const *out_
                                    int nranks, size_t count, int block,
                                    void *workspace, size_t workspace_bytes, int keep_trace,
                                    equarx_stream_t stream);
+
+/*
+ * The other flavours of the method, in the deep-pipelined form of
+ * equarx_allreduce_sim_pipelined (one persistent launch, one warp per
+ * 512-element tile, every message through the warp's staging FIFO and read
+ * back by the neighbouring lane).  `flavour` is a combination of:
+ *   EQUARX_FLAVOUR_SEMI_LOOP : semi-loop ring (Section 3.3, Fig. 5): shard k is
+ *       reduced by two half chains that meet at its owner,
+ *       A: k+N/2 -> k+N/2-1 -> ... -> k+1 -> k and B: k+N/2+1 -> ... -> k-1 -> k
+ *       (on 4 devices 2 -> 1 -> 0 and 3 -> 0, the paper's example); the owner
+ *       adds B's partial, then A's.  nranks must be even.  Without this bit:
+ *       the full-loop chain k+1 -> k+2 -> ... -> k.
+ *   EQUARX_FLAVOUR_QUANT_RS  : the reduce-scatter hops carry int8 records
+ *       (Section 3.1); without it they carry bf16 and every add is rounded to
+ *       bf16, as in the BF16 baseline.
+ *   EQUARX_FLAVOUR_QUANT_AG  : the reduced shard takes one more
+ *       quantize/dequantize pair (Section 3.4); without it the owner's sum is
+ *       rounded to bf16 and forwarded as is.
+ * QUANT_RS | QUANT_AG is equarx_allreduce_sim_pipelined's result bit for bit;
+ * 0 is the unquantized ring of equarx_allreduce_sim_bf16.
+ * Workspace: EQUARX_FLAVOUR_FIFO_BYTES of staging space, followed, with
+ * keep_trace, by a trace laid out as for equarx_allreduce_sim.  Events of a
+ * full loop: j = 0..N-2 the hops in chain order, N-1 the all-gather message;
+ * of a semi loop: 0..N/2-1 chain A's hops, N/2..N-2 chain B's hops, N-1 the
+ * all-gather message.  Events that the flavour does not quantize are zeroed.
+ * Other arguments and rules as for equarx_allreduce_sim.
+ */
+#define EQUARX_FLAVOUR_SEMI_LOOP 1
+#define EQUARX_FLAVOUR_QUANT_RS 2
+#define EQUARX_FLAVOUR_QUANT_AG 4
+#define EQUARX_FLAVOUR_FIFO_BYTES (16u * 1024u * 1024u)
+size_t equarx_allreduce_sim_flavour_workspace_bytes(int nranks, size_t count, int block, int flavour,
+                                                    int keep_trace);
+int equarx_allreduce_sim_flavour(const void *const *in_bf16, void *const *out_bf16,
+                                 int nranks, size_t count, int block, int flavour,
+                                 void *workspace, size_t workspace_bytes, int keep_trace,
+                                 equarx_stream_t stream);
 
 /* Workspace bytes of the unquantized comparator (two generations of bf16 messages: 4*count); 0 if invalid. */
 size_t equarx_allreduce_sim_bf16_workspace_bytes(int nranks, size_t count);

@@ -5,6 +5,9 @@ hand-written sm_100a kernels behind a C ABI (include/equarx.h); this package
 is the thin binding.  ``workloads`` holds the seeded synthetic inputs.
 """
 from .binding import (  # noqa: F401
+    FLAVOUR_QUANT_AG,
+    FLAVOUR_QUANT_RS,
+    FLAVOUR_SEMI_LOOP,
     EquarxError,
     LIB_PATH,
     MAX_RANKS,
@@ -12,6 +15,8 @@ from .binding import (  # noqa: F401
     allreduce_sim,
     allreduce_sim_bf16,
     allreduce_sim_bf16_workspace_bytes,
+    allreduce_sim_flavour,
+    allreduce_sim_flavour_workspace_bytes,
     allreduce_sim_pipelined,
     allreduce_sim_pipelined_workspace_bytes,
     allreduce_sim_range,

@@ -10,7 +10,10 @@ import ctypes
 from . import _build
 
 MAX_RANKS = 64
-OK, ERR_NULL, ERR_NRANKS, ERR_BLOCK, ERR_COUNT, ERR_ALIGN, ERR_WORKSPACE, ERR_ALIAS, ERR_CUDA, ERR_STATIC_LIMIT = range(10)
+(OK, ERR_NULL, ERR_NRANKS, ERR_BLOCK, ERR_COUNT, ERR_ALIGN, ERR_WORKSPACE, ERR_ALIAS, ERR_CUDA, ERR_STATIC_LIMIT,
+ ERR_FLAVOUR) = range(11)
+FLAVOUR_SEMI_LOOP, FLAVOUR_QUANT_RS, FLAVOUR_QUANT_AG = 1, 2, 4
+FLAVOUR_FIFO_BYTES = 16 * 1024 * 1024
 STATIC_WORKSPACE_BYTES = 16 * 1024 * 1024
 
 EXPORTS = (
@@ -19,6 +22,8 @@ EXPORTS = (
     "equarx_ag_dequant",
     "equarx_allreduce_sim_workspace_bytes",
     "equarx_allreduce_sim",
+    "equarx_allreduce_sim_flavour",
+    "equarx_allreduce_sim_flavour_workspace_bytes",
     "equarx_allreduce_sim_pipelined",
     "equarx_allreduce_sim_pipelined_workspace_bytes",
     "equarx_allreduce_sim_range",
@@ -50,6 +55,9 @@ def _load():
     lib.equarx_allreduce_sim_pipelined.argtypes = [vp, vp, ci, sz, ci, vp, sz, ci, vp]
     lib.equarx_allreduce_sim_pipelined_workspace_bytes.argtypes = [ci, sz, ci, ci]
     lib.equarx_allreduce_sim_pipelined_workspace_bytes.restype = sz
+    lib.equarx_allreduce_sim_flavour.argtypes = [vp, vp, ci, sz, ci, ci, vp, sz, ci, vp]
+    lib.equarx_allreduce_sim_flavour_workspace_bytes.argtypes = [ci, sz, ci, ci, ci]
+    lib.equarx_allreduce_sim_flavour_workspace_bytes.restype = sz
     lib.equarx_allreduce_sim_static.argtypes = [vp, vp, ci, sz, ci, vp]
     lib.equarx_allreduce_sim_bf16_workspace_bytes.argtypes = [ci, sz]
     lib.equarx_allreduce_sim_bf16_workspace_bytes.restype = sz
@@ -129,6 +137,17 @@ def allreduce_sim_pipelined(in_bf16, out_bf16, nranks, count, block, workspace, 
     _check(lib.equarx_allreduce_sim_pipelined(_table(in_bf16), _table(out_bf16), nranks, count, block,
                                               _ptr(workspace), workspace_bytes, int(bool(keep_trace)), _ptr(stream)),
            "equarx_allreduce_sim_pipelined")
+
+
+def allreduce_sim_flavour_workspace_bytes(nranks, count, block, flavour, keep_trace=False):
+    return lib.equarx_allreduce_sim_flavour_workspace_bytes(nranks, count, block, flavour, int(bool(keep_trace)))
+
+
+def allreduce_sim_flavour(in_bf16, out_bf16, nranks, count, block, flavour, workspace, workspace_bytes,
+                          keep_trace=False, stream=0):
+    _check(lib.equarx_allreduce_sim_flavour(_table(in_bf16), _table(out_bf16), nranks, count, block, flavour,
+                                            _ptr(workspace), workspace_bytes, int(bool(keep_trace)), _ptr(stream)),
+           "equarx_allreduce_sim_flavour")
 
 
 def allreduce_sim_range(in_bf16, out_bf16, nranks, count, block, workspace, workspace_bytes, keep_trace,

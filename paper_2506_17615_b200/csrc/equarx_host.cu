@@ -4,6 +4,7 @@
 // every entry point are in include/equarx.h.
 #include "equarx_kernels.cuh"
 
+#include <algorithm>
 #include <cstdlib>
 #include <cstring>
 
@@ -129,6 +130,20 @@ int check_tables(const void* const* in, void* const* out, int nranks, size_t byt
     return EQUARX_OK;
 }
 
+template <int LPB>
+const void* flavour_kernel_for(int flavour) {
+    switch (flavour) {
+        case 0: return reinterpret_cast<const void*>(flavour_kernel<LPB, false, false, false>);
+        case 1: return reinterpret_cast<const void*>(flavour_kernel<LPB, true, false, false>);
+        case 2: return reinterpret_cast<const void*>(flavour_kernel<LPB, false, true, false>);
+        case 3: return reinterpret_cast<const void*>(flavour_kernel<LPB, true, true, false>);
+        case 4: return reinterpret_cast<const void*>(flavour_kernel<LPB, false, false, true>);
+        case 5: return reinterpret_cast<const void*>(flavour_kernel<LPB, true, false, true>);
+        case 6: return reinterpret_cast<const void*>(flavour_kernel<LPB, false, true, true>);
+        default: return reinterpret_cast<const void*>(flavour_kernel<LPB, true, true, true>);
+    }
+}
+
 }  // namespace
 
 extern "C" {
@@ -144,6 +159,7 @@ const char* equarx_status_string(int status) {
         case EQUARX_ERR_WORKSPACE: return "EQUARX_ERR_WORKSPACE: workspace too small";
         case EQUARX_ERR_ALIAS: return "EQUARX_ERR_ALIAS: buffers overlap";
         case EQUARX_ERR_CUDA: return "EQUARX_ERR_CUDA: a kernel launch failed";
+        case EQUARX_ERR_FLAVOUR: return "EQUARX_ERR_FLAVOUR: flavour must be a combination of the EQUARX_FLAVOUR_* bits";
         case EQUARX_ERR_STATIC_LIMIT:
             return "EQUARX_ERR_STATIC_LIMIT: problem needs more than the 16 MiB built-in workspace";
         default: return "EQUARX: unknown status";
@@ -347,6 +363,87 @@ int equarx_allreduce_sim_pipelined(const void* const* in_bf16, void* const* out_
 
     void* params[1] = {&a};
     e = cudaLaunchKernel(kernel, dim3(unsigned(best_ctas)), dim3(kPipeThreads), params, 0, stream);
+    if (e != cudaSuccess) {
+        g_last_cuda_error = int(e);
+        (void)cudaGetLastError();
+        return EQUARX_ERR_CUDA;
+    }
+    return EQUARX_OK;
+}
+
+size_t equarx_allreduce_sim_flavour_workspace_bytes(int nranks, size_t count, int block, int flavour,
+                                                    int keep_trace) {
+    if (check_sim_shape(nranks, count, block) != EQUARX_OK) return 0;
+    if (flavour < 0 || flavour > 7) return 0;
+    if ((flavour & EQUARX_FLAVOUR_SEMI_LOOP) && nranks % 2 != 0) return 0;
+    size_t bytes = size_t(EQUARX_FLAVOUR_FIFO_BYTES);
+    if (keep_trace) bytes += equarx_allreduce_sim_workspace_bytes(nranks, count, block, 1);
+    return bytes;
+}
+
+int equarx_allreduce_sim_flavour(const void* const* in_bf16, void* const* out_bf16, int nranks, size_t count,
+                                 int block, int flavour, void* workspace, size_t workspace_bytes, int keep_trace,
+                                 equarx_stream_t stream) {
+    if (int st = check_sim_shape(nranks, count, block)) return st;
+    if (flavour < 0 || flavour > 7) return EQUARX_ERR_FLAVOUR;
+    if ((flavour & EQUARX_FLAVOUR_SEMI_LOOP) && nranks % 2 != 0) return EQUARX_ERR_NRANKS;
+    if (!workspace) return EQUARX_ERR_NULL;
+    const size_t need = equarx_allreduce_sim_flavour_workspace_bytes(nranks, count, block, flavour, keep_trace);
+    if (workspace_bytes < need) return EQUARX_ERR_WORKSPACE;
+    if (!aligned(workspace, 32)) return EQUARX_ERR_ALIGN;
+    if (int st = check_tables(in_bf16, out_bf16, nranks, 2 * count, workspace, need)) return st;
+
+    const uint32_t N = uint32_t(nranks);
+    const size_t shard = count / N;
+    FlavourArgs a = {};
+    a.neg_zero = -0.0f;
+    for (uint32_t r = 0; r < N; ++r) {
+        a.in[r] = in_bf16[r];
+        a.out[r] = out_bf16[r];
+    }
+    a.fifo = static_cast<char*>(workspace);
+    a.trace = keep_trace ? static_cast<char*>(workspace) + size_t(EQUARX_FLAVOUR_FIFO_BYTES) : nullptr;
+    a.shard = shard;
+    a.tiles_per_shard = (shard + kTileElems - 1) / kTileElems;
+    a.nranks = N;
+
+    const void* kernel = nullptr;
+    switch (block) {
+        case 64: kernel = flavour_kernel_for<4>(flavour); break;
+        case 128: kernel = flavour_kernel_for<8>(flavour); break;
+        case 256: kernel = flavour_kernel_for<16>(flavour); break;
+        default: kernel = flavour_kernel_for<32>(flavour); break;
+    }
+    int dev = 0, sms = 0, occ = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kPipeThreads, 0);
+    if (e != cudaSuccess || sms < 1 || occ < 1) {
+        g_last_cuda_error = int(e);
+        (void)cudaGetLastError();
+        return EQUARX_ERR_CUDA;
+    }
+    const uint64_t tiles = a.tiles_per_shard * N, wpc = kPipeThreads / 32;
+    uint64_t ctas = 0, best_rounds = ~uint64_t(0);
+    for (int c = 1; c <= occ; ++c) {                  // fewest rounds of tiles, then fewest CTAs
+        const uint64_t w = uint64_t(sms) * c * wpc, rounds = (tiles + w - 1) / w;
+        if (rounds < best_rounds) {
+            best_rounds = rounds;
+            ctas = uint64_t(sms) * c;
+        }
+    }
+    ctas = std::min<uint64_t>(ctas, (tiles + wpc - 1) / wpc);
+    ctas = std::min<uint64_t>(ctas, uint64_t(EQUARX_FLAVOUR_FIFO_BYTES) / (2 * kFifoEntryBytes) / wpc);
+    if (keep_trace) {                                  // events that this flavour does not quantize stay zero
+        e = cudaMemsetAsync(a.trace, 0, need - size_t(EQUARX_FLAVOUR_FIFO_BYTES), stream);
+        if (e != cudaSuccess) {
+            g_last_cuda_error = int(e);
+            (void)cudaGetLastError();
+            return EQUARX_ERR_CUDA;
+        }
+    }
+    void* params[1] = {&a};
+    e = cudaLaunchKernel(kernel, dim3(unsigned(ctas)), dim3(kPipeThreads), params, 0, stream);
     if (e != cudaSuccess) {
         g_last_cuda_error = int(e);
         (void)cudaGetLastError();

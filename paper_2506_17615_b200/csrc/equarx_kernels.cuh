@@ -94,6 +94,23 @@ __device__ __forceinline__ Vec8 ld_coherent_256(const void* p) {
     return r;
 }
 
+__device__ __forceinline__ Vec8 ld_fifo_256(const void* p) {
+    Vec8 r;
+    asm volatile("ld.global.L1::no_allocate.L2::evict_last.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r.w[0]), "=r"(r.w[1]), "=r"(r.w[2]), "=r"(r.w[3]),
+                   "=r"(r.w[4]), "=r"(r.w[5]), "=r"(r.w[6]), "=r"(r.w[7])
+                 : "l"(p)
+                 : "memory");
+    return r;
+}
+
+__device__ __forceinline__ void st_fifo_256(void* p, const Vec8& r) {
+    asm volatile("st.global.L1::no_allocate.L2::evict_last.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 ::"l"(p), "r"(r.w[0]), "r"(r.w[1]), "r"(r.w[2]), "r"(r.w[3]),
+                   "r"(r.w[4]), "r"(r.w[5]), "r"(r.w[6]), "r"(r.w[7])
+                 : "memory");
+}
+
 __device__ __forceinline__ uint4 ld_coherent_128(const void* p) {
     uint4 r;
     asm volatile("ld.global.cg.v4.b32 {%0,%1,%2,%3}, [%4];"
@@ -495,6 +512,202 @@ __global__ void __launch_bounds__(kPipeThreads, EQX_PIPE_MINBLOCKS) pipelined_ke
             // lane's load above has returned by then, because its value feeds the quantization of step j+1
         }
         __syncwarp();                                  // the next tile reuses the FIFO
+    }
+}
+
+// ---------------------------------------------------------------- the other flavours
+// Semi-loop ring (Section 3.3, Fig. 5) and stage selection (Section 3.4: quantize the
+// reduce-scatter, the all-gather, or both), in the same deep-pipelined form: one warp
+// carries a 512-element tile along its adder chain(s); every message goes through the
+// warp's two-entry staging FIFO and is read back by the neighbouring lane.  A message
+// is a 544-byte quantized record or, for an unquantized stage, 1024 bytes of bf16.
+constexpr int kFifoEntryBytes = 1024;
+
+struct FlavourArgs {
+    const void* in[kMaxRanks];
+    void* out[kMaxRanks];
+    char* fifo;                      // per-warp staging FIFOs (2 entries of kFifoEntryBytes)
+    char* trace;                     // record region [shard k][event j][tile], or nullptr
+    uint64_t shard;
+    uint64_t tiles_per_shard;
+    uint32_t nranks;
+    float neg_zero;
+};
+
+// One hop of a chain.  Sender side: the message of v (quantized record or bf16).  Receiver side
+// (the neighbouring lane): v_out = message (+) addend; with QUANT one fused multiply-add in fp32,
+// else an fp32 add rounded to bf16 (the BF16 baseline's hop).  `sub` is the lane's position in
+// the tile and flips with every hop.
+template <int LPB, bool QUANT>
+__device__ __forceinline__ void chain_hop(const float (&v)[16], const float (&addend)[16], float (&v_out)[16],
+                                          char* entry, char* trace_rec, uint32_t lane, uint32_t& sub, bool active,
+                                          float neg_zero) {
+    if (QUANT) {
+        uint4 codes;
+        float scale;
+        quantize_lane<LPB>(v, codes, scale, neg_zero);
+        const uint32_t d = (sub ^ lane) & 1u;                  // position p is held by lane p ^ d
+        float hdr = __shfl_sync(0xFFFFFFFFu, scale, ((lane * LPB) & 31u) ^ d);
+        if (lane >= 32u / LPB) hdr = 0.0f;
+        if (lane < 8) st_plain_f32(reinterpret_cast<float*>(entry) + lane, hdr);
+        if (active) st_plain_128(entry + kRecordHeader + sub * 16, codes);
+        if (trace_rec) {                                       // keep the message as well
+            if (lane < 8) st_plain_f32(reinterpret_cast<float*>(trace_rec) + lane, hdr);
+            if (active) st_plain_128(trace_rec + kRecordHeader + sub * 16, codes);
+        }
+        __syncwarp();
+        sub ^= 1u;
+        uint4 c = make_uint4(0, 0, 0, 0);
+        float s = 0.0f;
+        if (active) {
+            c = ld_coherent_128(entry + kRecordHeader + sub * 16);
+            s = ld_coherent_f32(reinterpret_cast<const float*>(entry) + sub / LPB);
+        }
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v_out[i] = addend[i];
+        dequant_add_x16(c, s, v_out);
+    } else {
+        Vec8 m;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) m.w[i] = pack_bf16x2_rn(v[2 * i], v[2 * i + 1]);
+        if (active) st_fifo_256(entry + sub * 32, m);
+        __syncwarp();
+        sub ^= 1u;
+        Vec8 r = {};
+        if (active) r = ld_fifo_256(entry + sub * 32);
+        float y[16];
+        widen_bf16x16(r, y);
+        Vec8 o;
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            o.w[i] = pack_bf16x2_rn(__fadd_rn(y[2 * i], addend[2 * i]), __fadd_rn(y[2 * i + 1], addend[2 * i + 1]));
+        widen_bf16x16(o, v_out);
+    }
+}
+
+template <int LPB, bool SEMI, bool QRS, bool QAG>
+__global__ void __launch_bounds__(kPipeThreads) flavour_kernel(const __grid_constant__ FlavourArgs a) {
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint64_t warps = (uint64_t)gridDim.x * (kPipeThreads / 32);
+    const uint64_t warp = (uint64_t)blockIdx.x * (kPipeThreads / 32) + (threadIdx.x >> 5);
+    const uint32_t N = a.nranks;
+    const uint32_t h = N / 2;
+    const uint64_t groups = a.shard >> 4;
+    const uint64_t tiles = a.tiles_per_shard * N;
+    char* const fifo = a.fifo + warp * (2 * kFifoEntryBytes);
+
+    for (uint64_t tile = warp; tile < tiles; tile += warps) {
+        const uint32_t k = (uint32_t)(tile / a.tiles_per_shard);
+        const uint64_t t = tile - (uint64_t)k * a.tiles_per_shard;
+        const bool active = t * 32 + lane < groups;
+        const uint64_t tile_off = (uint64_t)k * a.shard + t * kTileElems;        // first element of the tile
+        char* const trace0 = a.trace ? a.trace + ((uint64_t)k * N * a.tiles_per_shard + t) * kRecordBytes : nullptr;
+        uint32_t hops = 0;                                                       // FIFO entry = hops & 1
+
+        auto load_shard = [&](uint32_t rank, uint32_t pos, float (&dst)[16]) {
+            Vec8 x = {};
+            if (active) x = ld_coherent_256(static_cast<const char*>(a.in[rank % N]) + (tile_off + pos * 16) * 2);
+            widen_bf16x16(x, dst);
+        };
+        auto trace_of = [&](uint32_t event) -> char* {
+            return trace0 ? trace0 + (uint64_t)event * a.tiles_per_shard * kRecordBytes : nullptr;
+        };
+
+        float acc[16];                     // the owner's reduced tile
+        uint32_t sub;                      // this lane's position in the tile
+        if (!SEMI) {
+            sub = lane;
+            load_shard(k + 1, sub, acc);
+            for (uint32_t j = 1; j < N; ++j) {                                   // hop into rank k+1+j
+                float x[16];
+                load_shard(k + 1 + j, sub ^ 1u, x);
+                chain_hop<LPB, QRS>(acc, x, acc, fifo + (hops & 1u) * kFifoEntryBytes, QRS ? trace_of(j - 1) : nullptr,
+                                    lane, sub, active, a.neg_zero);
+                ++hops;
+            }
+        } else {
+            // chain B: k+h+1 -> ... -> k+N-1 -> owner (h-1 hops); starts at position `lane`
+            sub = lane;
+            const uint32_t acc_pos = lane ^ ((h - 1) & 1u);                      // position after B's hops
+            load_shard(k, h >= 2 ? acc_pos : lane, acc);
+            if (h >= 2) {
+                float v[16];
+                load_shard(k + h + 1, sub, v);
+                for (uint32_t j = 1; j < h; ++j) {
+                    char* entry = fifo + (hops & 1u) * kFifoEntryBytes;
+                    char* tr = QRS ? trace_of(h + j - 1) : nullptr;
+                    if (j + 1 < h) {
+                        float x[16];
+                        load_shard(k + h + 1 + j, sub ^ 1u, x);
+                        chain_hop<LPB, QRS>(v, x, v, entry, tr, lane, sub, active, a.neg_zero);
+                    } else {
+                        chain_hop<LPB, QRS>(v, acc, acc, entry, tr, lane, sub, active, a.neg_zero);
+                    }
+                    ++hops;
+                }
+            }
+            // chain A: k+h -> k+h-1 -> ... -> k+1 -> owner (h hops); starts so that it ends on acc's position
+            sub = (h >= 2 ? acc_pos : lane) ^ (h & 1u);
+            float v[16];
+            load_shard(k + h, sub, v);
+            for (uint32_t j = 1; j <= h; ++j) {
+                char* entry = fifo + (hops & 1u) * kFifoEntryBytes;
+                char* tr = QRS ? trace_of(j - 1) : nullptr;
+                if (j < h) {
+                    float x[16];
+                    load_shard(k + h - j, sub ^ 1u, x);
+                    chain_hop<LPB, QRS>(v, x, v, entry, tr, lane, sub, active, a.neg_zero);
+                } else {
+                    chain_hop<LPB, QRS>(v, acc, acc, entry, tr, lane, sub, active, a.neg_zero);
+                }
+                ++hops;
+            }
+        }
+
+        // all-gather: one more message, quantized or bf16, dequantized/forwarded to every rank
+        Vec8 o;
+        {
+            char* entry = fifo + (hops & 1u) * kFifoEntryBytes;
+            if (QAG) {
+                uint4 codes;
+                float scale;
+                quantize_lane<LPB>(acc, codes, scale, a.neg_zero);
+                const uint32_t d = (sub ^ lane) & 1u;
+                float hdr = __shfl_sync(0xFFFFFFFFu, scale, ((lane * LPB) & 31u) ^ d);
+                if (lane >= 32u / LPB) hdr = 0.0f;
+                char* tr = trace_of(N - 1);
+                if (lane < 8) st_plain_f32(reinterpret_cast<float*>(entry) + lane, hdr);
+                if (active) st_plain_128(entry + kRecordHeader + sub * 16, codes);
+                if (tr) {
+                    if (lane < 8) st_plain_f32(reinterpret_cast<float*>(tr) + lane, hdr);
+                    if (active) st_plain_128(tr + kRecordHeader + sub * 16, codes);
+                }
+                __syncwarp();
+                sub ^= 1u;
+                uint4 c = make_uint4(0, 0, 0, 0);
+                float s = 0.0f;
+                if (active) {
+                    c = ld_coherent_128(entry + kRecordHeader + sub * 16);
+                    s = ld_coherent_f32(reinterpret_cast<const float*>(entry) + sub / LPB);
+                }
+                o = dequant_to_bf16x16(c, s);
+            } else {
+                Vec8 m;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) m.w[i] = pack_bf16x2_rn(acc[2 * i], acc[2 * i + 1]);
+                if (active) st_fifo_256(entry + sub * 32, m);
+                __syncwarp();
+                sub ^= 1u;
+                o = Vec8{};
+                if (active) o = ld_fifo_256(entry + sub * 32);
+            }
+            ++hops;
+        }
+        if (active) {
+            const uint64_t byte_off = (tile_off + sub * 16) * 2;
+            for (uint32_t r = 0; r < N; ++r) st_stream_256(static_cast<char*>(a.out[r]) + byte_off, o);
+        }
+        __syncwarp();                      // the next tile reuses the FIFO
     }
 }
 
