@@ -363,6 +363,20 @@ def main():
                 "frac_of_nominal_8TBs": steps_gbs / NOMINAL_HBM_GBS, "kernels": kernels,
                 "hop_traffic_bytes_per_launch": DAR_TRAFFIC_BYTES_PER_ELEMENT * count}
 
+    # ---- the other flavours (semi-loop ring, stage selection), same workload, pipelined form
+    flavours = {}
+    wbf = eq.allreduce_sim_flavour_workspace_bytes(N, count, block, 7 if N % 2 == 0 else 6, False)
+    wsf = torch.empty(wbf, dtype=torch.uint8, device=dev)
+    names = {0: "full_loop_unquantized", 2: "full_loop_rs_only", 4: "full_loop_ag_only", 6: "full_loop_rs_ag",
+             1: "semi_loop_unquantized", 3: "semi_loop_rs_only", 5: "semi_loop_ag_only", 7: "semi_loop_rs_ag"}
+    for fl, name in sorted(names.items()):
+        if (fl & 1) and N % 2:
+            continue
+        ms_f = timed(lambda i, fl=fl: eq.allreduce_sim_flavour(ins[i % sets], outs[i % sets], N, count, block, fl,
+                                                               wsf, wbf, False, stream), max(5, min(200, args.steps)))
+        flavours[name] = {"ms_per_step": ms_f, "value": aggregate_value(in_bytes, ms_f, world), "unit": UNIT}
+    del wsf
+
     # unquantized comparator on the same GPU, same inputs
     wb16 = eq.allreduce_sim_bf16_workspace_bytes(N, count)
     ws16 = torch.empty(wb16, dtype=torch.uint8, device=dev)
@@ -382,35 +396,38 @@ def main():
                 "frac_of_measured_peak": count * (8 * N - 4) / (ms16 * 1e-3) / 1e9 / peak}
     del ws16
 
-    # end to end: pinned host buffers, copies inside the timed region
+    # end to end through the host-buffer front end: every step uploads its N input tensors from
+    # pinned host memory, runs the AllReduce and downloads the N outputs; copies of neighbouring
+    # steps overlap with the kernels (three streams, two device buffer sets)
     e2e = None
     if not args.no_e2e:
-        h_in = torch.empty((N, count), dtype=torch.bfloat16).pin_memory()
-        h_in.copy_(torch.stack(ins[0]).cpu())
-        h_out = torch.empty((N, count), dtype=torch.bfloat16).pin_memory()
-        d_in = torch.empty((N, count), dtype=torch.bfloat16, device=dev)
-        d_out = torch.empty((N, count), dtype=torch.bfloat16, device=dev)
-        d_ins, d_outs = [d_in[r] for r in range(N)], [d_out[r] for r in range(N)]
-
-        def e2e_step():
-            d_in.copy_(h_in, non_blocking=True)
-            eq.allreduce_sim_pipelined(d_ins, d_outs, N, count, block, wsp, wbp, False, stream)
-            h_out.copy_(d_out, non_blocking=True)
-
+        from paper_2506_17615_b200.host_api import HostPipeline
+        h_in = [torch.empty((N, count), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
+        for i, h in enumerate(h_in):
+            h.copy_(torch.stack(ins[i % sets]).cpu())
+        h_out = [torch.empty((N, count), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
+        pipe = HostPipeline(N, count, block, dev)
         e_steps = max(3, min(20, args.steps))
-        for _ in range(3):
-            e2e_step()
+        for i in range(3):
+            pipe.submit(h_in[i % 2], h_out[i % 2])
+        pipe.wait()
         barrier()
-        ev0.record()
-        for _ in range(e_steps):
-            e2e_step()
-        ev1.record()
+        t0 = torch.cuda.Event(enable_timing=True)
+        t1 = torch.cuda.Event(enable_timing=True)
+        t0.record()
+        pipe.h2d.wait_event(t0)
+        for i in range(e_steps):
+            pipe.submit(h_in[i % 2], h_out[i % 2])
+        torch.cuda.current_stream().wait_stream(pipe.d2h)
+        torch.cuda.current_stream().wait_stream(pipe.comp)
+        t1.record()
         torch.cuda.synchronize()
         barrier()
-        ms_e = max_over_ranks(ev0.elapsed_time(ev1), world, dev) / e_steps
+        ms_e = max_over_ranks(t0.elapsed_time(t1), world, dev) / e_steps
         e2e = {"value": aggregate_value(in_bytes, ms_e, world), "unit": UNIT, "h2d_bytes_per_step": in_bytes,
-               "d2h_bytes_per_step": in_bytes, "ms_per_step": ms_e, "steps": e_steps}
-        del h_in, h_out, d_in, d_out
+               "d2h_bytes_per_step": in_bytes, "ms_per_step": ms_e, "steps": e_steps,
+               "api": "paper_2506_17615_b200.host_api.HostPipeline.submit (copies overlapped across steps)"}
+        del h_in, h_out, pipe
 
     sampler.stop()
     clocks = sampler.summary(windows)
@@ -427,7 +444,7 @@ def main():
                        "pdl_between_step_launches": os.environ.get("EQUARX_PDL", "1") != "0"},
             "e2e": e2e, "gpu_launches": args.steps, "clocks": clocks,
             "roofline": roofline, "schedule": "pipelined (equarx_allreduce_sim_pipelined, 1 launch per step)",
-            "by_steps": by_steps, "bf16_sim": bf16_sim,
+            "by_steps": by_steps, "flavours": flavours, "bf16_sim": bf16_sim,
             "speedup_vs_bf16_sim": value / world / bf16_sim["value"],
         }
         if world == 1 and not args.no_cpu_baseline:

@@ -264,3 +264,20 @@ def test_sweep_points_large_sampled(gu, nranks, block, dist, nbytes):
         gu.assert_same_words(gu.gather_blocks(out, picks, block), exp, f"{variant} {w.name}")
         del out
     torch.cuda.empty_cache()
+
+
+def test_host_pipeline_matches_device_path(gu):
+    """The host-buffer front end (pinned memory in, pinned memory out, overlapped copies) returns
+    the same bits as the device-resident call, for several submissions in flight."""
+    from paper_2506_17615_b200.host_api import HostPipeline
+    w = wl.Workload("t", 4, 4 * 256 * 40, 256, "normal", seed=1)
+    pipe = HostPipeline(w.nranks, w.count, w.block)
+    xs = [wl.make_inputs(wl.Workload("t", 4, w.count, 256, "normal", seed=s)) for s in range(5)]
+    h_in = [x.pin_memory() for x in xs]
+    h_out = [torch.empty_like(x).pin_memory() for x in xs]
+    for i in range(5):
+        pipe.submit(h_in[i], h_out[i])
+    pipe.wait()
+    for i in range(5):
+        exp = oracle.allreduce(wl.as_u16(xs[i]), 256)["out"]
+        gu.assert_same_words(h_out[i], exp, f"submission {i}")
