@@ -460,6 +460,21 @@ __global__ void __launch_bounds__(kPipeThreads, EQX_PIPE_MINBLOCKS) pipelined_ke
     const uint64_t tiles = a.tiles_per_shard * N;
     char* const fifo = a.records + warp * (2 * kRecordBytes);
 
+    // the first shard of a tile is fetched while the previous tile finishes (its last step needs
+    // no prefetch of its own, so the same registers are free)
+    auto first_shard = [&](uint64_t tile_) {
+        Vec8 x = {};
+        if (tile_ < tiles) {
+            const uint32_t k_ = (uint32_t)(tile_ / a.tiles_per_shard);
+            const uint64_t t_ = tile_ - (uint64_t)k_ * a.tiles_per_shard;
+            const uint32_t rho_ = k_ + 1 == N ? 0 : k_ + 1;
+            if (t_ * 32 + lane < groups)
+                x = ld_coherent_256(static_cast<const char*>(a.in[rho_]) + ((uint64_t)k_ * a.shard + (t_ * 32 + lane) * 16) * 2);
+        }
+        return x;
+    };
+    Vec8 xw = first_shard(warp);
+
     for (uint64_t tile = warp; tile < tiles; tile += warps) {
         const uint32_t k = (uint32_t)(tile / a.tiles_per_shard);           // shard
         const uint64_t t = tile - (uint64_t)k * a.tiles_per_shard;
@@ -469,15 +484,17 @@ __global__ void __launch_bounds__(kPipeThreads, EQX_PIPE_MINBLOCKS) pipelined_ke
         char* const trace = a.records + ((uint64_t)k * N * a.tiles_per_shard + t) * kRecordBytes;
 
         uint32_t rho = k + 1 == N ? 0 : k + 1;         // rank of step 0
-        Vec8 xw = {};
-        if (active) xw = ld_coherent_256(static_cast<const char*>(a.in[rho]) + (shard_off + g * 16) * 2);
         float v[16];
         widen_bf16x16(xw, v);
         uint32_t sub = lane;                           // position inside the tile handled at step j
         for (uint32_t j = 0;; ++j) {
             rho = rho + 1 == N ? 0 : rho + 1;
-            if (active && j + 1 < N)                   // the next step's bf16 shard arrives while this step computes
-                xw = ld_coherent_256(static_cast<const char*>(a.in[rho]) + (shard_off + (t * 32 + (sub ^ 1)) * 16) * 2);
+            if (j + 1 < N) {                           // the next step's bf16 shard arrives while this step computes
+                if (active)
+                    xw = ld_coherent_256(static_cast<const char*>(a.in[rho]) + (shard_off + (t * 32 + (sub ^ 1)) * 16) * 2);
+            } else {
+                xw = first_shard(tile + warps);        // last step: fetch the next tile's first shard instead
+            }
             uint4 codes;
             float scale;
             quantize_lane<LPB>(v, codes, scale, a.neg_zero);
