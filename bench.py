@@ -368,7 +368,8 @@ def main():
     wbf = eq.allreduce_sim_flavour_workspace_bytes(N, count, block, 7 if N % 2 == 0 else 6, False)
     wsf = torch.empty(wbf, dtype=torch.uint8, device=dev)
     names = {0: "full_loop_unquantized", 2: "full_loop_rs_only", 4: "full_loop_ag_only", 6: "full_loop_rs_ag",
-             1: "semi_loop_unquantized", 3: "semi_loop_rs_only", 5: "semi_loop_ag_only", 7: "semi_loop_rs_ag"}
+             1: "semi_loop_unquantized", 3: "semi_loop_rs_only", 5: "semi_loop_ag_only", 7: "semi_loop_rs_ag",
+             6 | 8: "full_loop_rs_ag_fp8_e4m3", 6 | 16: "full_loop_rs_ag_fp8_e5m2"}
     for fl, name in sorted(names.items()):
         if (fl & 1) and N % 2:
             continue

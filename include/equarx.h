@@ -198,6 +198,14 @@ int equarx_allreduce_sim_pipelined(const void *const *in_bf16, void *const *out_
  *   EQUARX_FLAVOUR_QUANT_AG  : the reduced shard takes one more
  *       quantize/dequantize pair (Section 3.4); without it the owner's sum is
  *       rounded to bf16 and forwarded as is.
+ *   EQUARX_FLAVOUR_E4M3, EQUARX_FLAVOUR_E5M2 (at most one, and only with a
+ *       quantized stage): the payload is FP8 instead of int8 (Section 4 names
+ *       all three).  Same rule with the format's largest finite value in place
+ *       of 127: scale = amax/448 (E4M3, bias 7, no infinities) or amax/57344
+ *       (E5M2, bias 15), code = fp8_rne(v * (FMAX/amax)) saturating at +-FMAX;
+ *       blocks with amax < 2^-117 (E4M3) or 2^-110 (E5M2) get scale 0 and zero
+ *       codes.  FP8 has a negative zero, so a flushed negative input comes back
+ *       as -0.0.  The codes of a trace are the raw FP8 bytes.
  * QUANT_RS | QUANT_AG is equarx_allreduce_sim_pipelined's result bit for bit;
  * 0 is the unquantized ring of equarx_allreduce_sim_bf16.
  * Workspace: EQUARX_FLAVOUR_FIFO_BYTES of staging space, followed, with
@@ -210,6 +218,8 @@ int equarx_allreduce_sim_pipelined(const void *const *in_bf16, void *const *out_
 #define EQUARX_FLAVOUR_SEMI_LOOP 1
 #define EQUARX_FLAVOUR_QUANT_RS 2
 #define EQUARX_FLAVOUR_QUANT_AG 4
+#define EQUARX_FLAVOUR_E4M3 8
+#define EQUARX_FLAVOUR_E5M2 16
 #define EQUARX_FLAVOUR_FIFO_BYTES (16u * 1024u * 1024u)
 size_t equarx_allreduce_sim_flavour_workspace_bytes(int nranks, size_t count, int block, int flavour,
                                                     int keep_trace);

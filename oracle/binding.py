@@ -50,7 +50,7 @@ def _load():
         lib.equarx_oracle_ag_dequant.argtypes = [vp, vp, sz, ci, vp]
         lib.equarx_oracle_allreduce.argtypes = [vp, vp, ci, sz, ci, vp, vp, vp]
         lib.equarx_oracle_allreduce_bf16.argtypes = [vp, vp, ci, sz]
-        lib.equarx_oracle_allreduce_variant.argtypes = [vp, vp, ci, sz, ci, ci, ci, ci, vp, vp]
+        lib.equarx_oracle_allreduce_variant.argtypes = [vp, vp, ci, sz, ci, ci, ci, ci, ci, vp, vp]
         lib.equarx_oracle_error_bound.argtypes = [vp, vp, ci, sz, ci, vp]
         for name in ("quantize_blocks", "rs_step", "ag_dequant", "allreduce",
                      "allreduce_bf16", "error_bound", "allreduce_variant"):
@@ -147,9 +147,14 @@ def allreduce(inputs_bf16, block, trace=False, exact=False):
     return res
 
 
-def allreduce_variant(inputs_bf16, block, semi_loop=False, quant_rs=True, quant_ag=True, trace=False):
+PAYLOADS = {"int8": 0, "e4m3": 1, "e5m2": 2}
+
+
+def allreduce_variant(inputs_bf16, block, semi_loop=False, quant_rs=True, quant_ag=True, trace=False,
+                      payload="int8"):
     """The flavours of Sections 3.3 / 3.4: full-loop or semi-loop ring, with the reduce-scatter
-    hops and/or the all-gather quantized.  Returns a dict like allreduce()."""
+    hops and/or the all-gather quantized, int8 or FP8 payload.  Returns a dict like allreduce();
+    trace codes are the raw payload bytes."""
     x = _arr(inputs_bf16, np.uint16)
     n_ranks, count = x.shape
     if block < 1:
@@ -165,7 +170,7 @@ def allreduce_variant(inputs_bf16, block, semi_loop=False, quant_rs=True, quant_
         res["scales"], res["codes"] = ts, tc
     _check(_load().equarx_oracle_allreduce_variant(
         _ptr_array([x[r] for r in range(n_ranks)]), _ptr_array([out[r] for r in range(n_ranks)]),
-        n_ranks, count, block, int(semi_loop), int(quant_rs), int(quant_ag),
+        n_ranks, count, block, int(semi_loop), int(quant_rs), int(quant_ag), PAYLOADS[payload],
         _p(ts) if trace else None, _p(tc) if trace else None), "allreduce_variant")
     return res
 

@@ -115,6 +115,94 @@ static void quantize_one_block(const float *v, int block, int8_t *code, float *s
     *scale_out = scale;
 }
 
+/*
+ * FP8 payloads (Section 4: "int8, FP8 (E4M3) and FP8 (E5M2), and it uses symmetric
+ * quantization").  Reading: the same block-wise rule with the format's largest finite
+ * value in place of 127: scale = amax / FMAX, code = fp8_rne(v * (FMAX / amax)),
+ * saturating at +-FMAX; E4M3 is the 8-bit format with bias 7, no infinities and
+ * FMAX = 448, E5M2 the one with bias 15 and FMAX = 57344.  Blocks with
+ * amax < FMAX_pow2 * 2^-126 (2^-117 for E4M3, 2^-110 for E5M2) get scale 0 and zero
+ * codes, which keeps the scale normal and FMAX / amax finite.
+ */
+typedef struct { int p; int emin; int bias; float fmax; float flush; } fp8_format;
+static const fp8_format FP8_E4M3 = {4, -6, 7, 448.0f, 0x1p-117f};
+static const fp8_format FP8_E5M2 = {3, -14, 15, 57344.0f, 0x1p-110f};
+
+/* round t to the nearest value of the format (ties to even), saturating at +-fmax */
+static float fp8_round(float t, const fp8_format *f)
+{
+    if (t == 0.0f) return t;
+    float a = fabsf(t);
+    int e;
+    (void)frexpf(a, &e);                 /* a = m * 2^e, m in [0.5, 1): floor(log2 a) = e - 1 */
+    int E = e - 1;
+    if (E < f->emin) E = f->emin;        /* subnormals share the spacing of emin */
+    float ulp = ldexpf(1.0f, E - (f->p - 1));
+    float r = rintf(a / ulp) * ulp;      /* both scalings are by powers of two: exact */
+    if (r > f->fmax) r = f->fmax;
+    return copysignf(r, t);
+}
+
+/* the byte that encodes a value of the format: sign, exponent field, p-1 mantissa bits */
+static uint8_t fp8_encode(float r, const fp8_format *f)
+{
+    uint8_t sign = signbit(r) ? 0x80u : 0u;
+    float a = fabsf(r);
+    if (a == 0.0f) return sign;
+    int e;
+    (void)frexpf(a, &e);
+    int E = e - 1;
+    unsigned field, mant;
+    if (E < f->emin) {
+        field = 0;
+        mant = (unsigned)(a / ldexpf(1.0f, f->emin - (f->p - 1)));
+    } else {
+        field = (unsigned)(E + f->bias);
+        mant = (unsigned)((a / ldexpf(1.0f, E) - 1.0f) * (float)(1 << (f->p - 1)));
+    }
+    return (uint8_t)(sign | (field << (f->p - 1)) | mant);
+}
+
+static float fp8_decode(uint8_t byte, const fp8_format *f)
+{
+    unsigned field = (byte & 0x7Fu) >> (f->p - 1);
+    unsigned mant = byte & ((1u << (f->p - 1)) - 1u);
+    float a = field == 0 ? (float)mant * ldexpf(1.0f, f->emin - (f->p - 1))
+                         : (1.0f + (float)mant / (float)(1 << (f->p - 1))) * ldexpf(1.0f, (int)field - f->bias);
+    return (byte & 0x80u) ? -a : a;
+}
+
+/* payload: 0 int8, 1 FP8 E4M3, 2 FP8 E5M2.  Codes are stored as raw bytes. */
+static void quantize_one_block_payload(const float *v, int block, int payload, int8_t *code, float *scale_out)
+{
+    if (payload == 0) {
+        quantize_one_block(v, block, code, scale_out);
+        return;
+    }
+    const fp8_format *f = payload == 1 ? &FP8_E4M3 : &FP8_E5M2;
+    float amax = 0.0f;
+    for (int i = 0; i < block; ++i) {
+        float a = fabsf(v[i]);
+        if (a > amax) amax = a;
+    }
+    float scale, inv;
+    if (!(amax >= f->flush)) {
+        scale = 0.0f;
+        inv = 0.0f;
+    } else {
+        scale = amax / f->fmax;
+        inv = f->fmax / amax;
+    }
+    for (int i = 0; i < block; ++i) code[i] = (int8_t)fp8_encode(fp8_round(v[i] * inv, f), f);
+    *scale_out = scale;
+}
+
+static float code_value(int8_t code, int payload)
+{
+    if (payload == 0) return (float)code;
+    return fp8_decode((uint8_t)code, payload == 1 ? &FP8_E4M3 : &FP8_E5M2);
+}
+
 static int check_block_count(size_t count, int block)
 {
     if (block < 1) return ORACLE_ERR_BLOCK;
@@ -361,15 +449,15 @@ int equarx_oracle_allreduce_bf16(const uint16_t *const *in, uint16_t *const *out
  *   semi loop : j = 0..N/2-1 chain A's hops, j = N/2..N-2 chain B's hops, j = N-1
  *               the all-gather message.
  * Events that are not quantized in the chosen flavour are left zero.
+ * payload: 0 int8, 1 FP8 E4M3, 2 FP8 E5M2 (codes are the raw bytes).
  */
-static void hop_receive(int quant, const float *v_sent, int block, const float *addend,
-                        int addend_is_bf16_exact, float *v_out, int8_t *codes, float *scale)
+static void hop_receive(int quant, int payload, const float *v_sent, int block, const float *addend,
+                        float *v_out, int8_t *codes, float *scale)
 {
     /* sender side: message of v_sent; receiver side: v_out = message (+) addend */
-    (void)addend_is_bf16_exact;
     if (quant) {
-        quantize_one_block(v_sent, block, codes, scale);
-        for (int i = 0; i < block; ++i) v_out[i] = fmaf((float)codes[i], *scale, addend[i]);
+        quantize_one_block_payload(v_sent, block, payload, codes, scale);
+        for (int i = 0; i < block; ++i) v_out[i] = fmaf(code_value(codes[i], payload), *scale, addend[i]);
     } else {
         for (int i = 0; i < block; ++i) {
             float msg = bf16_to_f32(f32_to_bf16_rne(v_sent[i]));      /* the bf16 message */
@@ -380,13 +468,14 @@ static void hop_receive(int quant, const float *v_sent, int block, const float *
 
 int equarx_oracle_allreduce_variant(const uint16_t *const *in, uint16_t *const *out,
                                     int nranks, size_t count, int block,
-                                    int semi_loop, int quant_rs, int quant_ag,
+                                    int semi_loop, int quant_rs, int quant_ag, int payload,
                                     float *trace_scales, int8_t *trace_codes)
 {
     if (!in || !out) return ORACLE_ERR_NULL;
     int st = check_sim_args(nranks, count, block);
     if (st) return st;
     if (semi_loop && (nranks % 2 != 0)) return ORACLE_ERR_NRANKS;
+    if (payload < 0 || payload > 2) return ORACLE_ERR_BLOCK;
     const size_t N = (size_t)nranks;
     const size_t shard = count / N;
     const size_t bps = shard / (size_t)block;
@@ -417,7 +506,7 @@ int equarx_oracle_allreduce_variant(const uint16_t *const *in, uint16_t *const *
                 LOAD(v, k + 1);
                 for (size_t j = 1; j < N; ++j) {           /* hop into rank k+1+j */
                     LOAD(x, k + 1 + j);
-                    hop_receive(quant_rs, v, block, x, 1, w, codes, &scale);
+                    hop_receive(quant_rs, payload, v, block, x, w, codes, &scale);
                     memcpy(v, w, (size_t)block * sizeof(float));
                     RECORD(quant_rs);
                 }
@@ -433,7 +522,7 @@ int equarx_oracle_allreduce_variant(const uint16_t *const *in, uint16_t *const *
                         const int last = (j == h - 1);
                         if (!last) LOAD(x, k + h + 1 + j);
                         event = event_b++;
-                        hop_receive(quant_rs, v, block, last ? acc : x, 1, w, codes, &scale);
+                        hop_receive(quant_rs, payload, v, block, last ? acc : x, w, codes, &scale);
                         RECORD(quant_rs);
                         memcpy(last ? acc : v, w, (size_t)block * sizeof(float));
                     }
@@ -444,7 +533,7 @@ int equarx_oracle_allreduce_variant(const uint16_t *const *in, uint16_t *const *
                 for (size_t j = 1; j <= h; ++j) {
                     const int last = (j == h);
                     if (!last) LOAD(x, k + h - j);
-                    hop_receive(quant_rs, v, block, last ? acc : x, 1, w, codes, &scale);
+                    hop_receive(quant_rs, payload, v, block, last ? acc : x, w, codes, &scale);
                     RECORD(quant_rs);
                     memcpy(last ? acc : v, w, (size_t)block * sizeof(float));
                 }
@@ -452,10 +541,10 @@ int equarx_oracle_allreduce_variant(const uint16_t *const *in, uint16_t *const *
             /* acc is the owner's reduced block: fp32 if the hops were quantized, else a bf16 value */
             event = N - 1;
             if (quant_ag) {
-                quantize_one_block(acc, block, codes, &scale);
+                quantize_one_block_payload(acc, block, payload, codes, &scale);
                 RECORD(1);
                 for (int i = 0; i < block; ++i) {
-                    uint16_t h16 = f32_to_bf16_rne((float)codes[i] * scale);
+                    uint16_t h16 = f32_to_bf16_rne(code_value(codes[i], payload) * scale);
                     for (size_t r = 0; r < N; ++r) out[r][base + (size_t)i] = h16;
                 }
             } else {

@@ -5,6 +5,8 @@ hand-written sm_100a kernels behind a C ABI (include/equarx.h); this package
 is the thin binding.  ``workloads`` holds the seeded synthetic inputs.
 """
 from .binding import (  # noqa: F401
+    FLAVOUR_E4M3,
+    FLAVOUR_E5M2,
     FLAVOUR_QUANT_AG,
     FLAVOUR_QUANT_RS,
     FLAVOUR_SEMI_LOOP,

@@ -12,7 +12,7 @@ from . import _build
 MAX_RANKS = 64
 (OK, ERR_NULL, ERR_NRANKS, ERR_BLOCK, ERR_COUNT, ERR_ALIGN, ERR_WORKSPACE, ERR_ALIAS, ERR_CUDA, ERR_STATIC_LIMIT,
  ERR_FLAVOUR) = range(11)
-FLAVOUR_SEMI_LOOP, FLAVOUR_QUANT_RS, FLAVOUR_QUANT_AG = 1, 2, 4
+FLAVOUR_SEMI_LOOP, FLAVOUR_QUANT_RS, FLAVOUR_QUANT_AG, FLAVOUR_E4M3, FLAVOUR_E5M2 = 1, 2, 4, 8, 16
 FLAVOUR_FIFO_BYTES = 16 * 1024 * 1024
 STATIC_WORKSPACE_BYTES = 16 * 1024 * 1024
 

@@ -130,18 +130,36 @@ int check_tables(const void* const* in, void* const* out, int nranks, size_t byt
     return EQUARX_OK;
 }
 
+template <int LPB, int PAYLOAD>
+const void* flavour_kernel_for(int flavour) {
+    switch (flavour & 7) {
+        case 2: return reinterpret_cast<const void*>(flavour_kernel<LPB, false, true, false, PAYLOAD>);
+        case 3: return reinterpret_cast<const void*>(flavour_kernel<LPB, true, true, false, PAYLOAD>);
+        case 4: return reinterpret_cast<const void*>(flavour_kernel<LPB, false, false, true, PAYLOAD>);
+        case 5: return reinterpret_cast<const void*>(flavour_kernel<LPB, true, false, true, PAYLOAD>);
+        case 6: return reinterpret_cast<const void*>(flavour_kernel<LPB, false, true, true, PAYLOAD>);
+        case 7: return reinterpret_cast<const void*>(flavour_kernel<LPB, true, true, true, PAYLOAD>);
+        // nothing is quantized: the payload type does not matter
+        case 1: return reinterpret_cast<const void*>(flavour_kernel<LPB, true, false, false, 1>);
+        default: return reinterpret_cast<const void*>(flavour_kernel<LPB, false, false, false, 1>);
+    }
+}
+
 template <int LPB>
 const void* flavour_kernel_for(int flavour) {
-    switch (flavour) {
-        case 0: return reinterpret_cast<const void*>(flavour_kernel<LPB, false, false, false>);
-        case 1: return reinterpret_cast<const void*>(flavour_kernel<LPB, true, false, false>);
-        case 2: return reinterpret_cast<const void*>(flavour_kernel<LPB, false, true, false>);
-        case 3: return reinterpret_cast<const void*>(flavour_kernel<LPB, true, true, false>);
-        case 4: return reinterpret_cast<const void*>(flavour_kernel<LPB, false, false, true>);
-        case 5: return reinterpret_cast<const void*>(flavour_kernel<LPB, true, false, true>);
-        case 6: return reinterpret_cast<const void*>(flavour_kernel<LPB, false, true, true>);
-        default: return reinterpret_cast<const void*>(flavour_kernel<LPB, true, true, true>);
-    }
+    if (flavour & EQUARX_FLAVOUR_E4M3) return flavour_kernel_for<LPB, 2>(flavour);
+    if (flavour & EQUARX_FLAVOUR_E5M2) return flavour_kernel_for<LPB, 3>(flavour);
+    return flavour_kernel_for<LPB, 1>(flavour);
+}
+
+// a valid flavour: any of the three schedule bits, at most one payload bit, and a payload bit
+// only together with a quantized stage
+inline bool flavour_ok(int flavour) {
+    if (flavour < 0 || flavour > 31) return false;
+    const bool e4 = flavour & EQUARX_FLAVOUR_E4M3, e5 = flavour & EQUARX_FLAVOUR_E5M2;
+    if (e4 && e5) return false;
+    if ((e4 || e5) && !(flavour & (EQUARX_FLAVOUR_QUANT_RS | EQUARX_FLAVOUR_QUANT_AG))) return false;
+    return true;
 }
 
 }  // namespace
@@ -374,7 +392,7 @@ int equarx_allreduce_sim_pipelined(const void* const* in_bf16, void* const* out_
 size_t equarx_allreduce_sim_flavour_workspace_bytes(int nranks, size_t count, int block, int flavour,
                                                     int keep_trace) {
     if (check_sim_shape(nranks, count, block) != EQUARX_OK) return 0;
-    if (flavour < 0 || flavour > 7) return 0;
+    if (!flavour_ok(flavour)) return 0;
     if ((flavour & EQUARX_FLAVOUR_SEMI_LOOP) && nranks % 2 != 0) return 0;
     size_t bytes = size_t(EQUARX_FLAVOUR_FIFO_BYTES);
     if (keep_trace) bytes += equarx_allreduce_sim_workspace_bytes(nranks, count, block, 1);
@@ -385,7 +403,7 @@ int equarx_allreduce_sim_flavour(const void* const* in_bf16, void* const* out_bf
                                  int block, int flavour, void* workspace, size_t workspace_bytes, int keep_trace,
                                  equarx_stream_t stream) {
     if (int st = check_sim_shape(nranks, count, block)) return st;
-    if (flavour < 0 || flavour > 7) return EQUARX_ERR_FLAVOUR;
+    if (!flavour_ok(flavour)) return EQUARX_ERR_FLAVOUR;
     if ((flavour & EQUARX_FLAVOUR_SEMI_LOOP) && nranks % 2 != 0) return EQUARX_ERR_NRANKS;
     if (!workspace) return EQUARX_ERR_NULL;
     const size_t need = equarx_allreduce_sim_flavour_workspace_bytes(nranks, count, block, flavour, keep_trace);

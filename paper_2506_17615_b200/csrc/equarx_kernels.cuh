@@ -286,6 +286,106 @@ __device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
     return d;
 }
 
+// ---------------------------------------------------------------- FP8 payloads
+// The same block-wise rule with the format's largest finite value in place of 127
+// (E4M3: 448, E5M2: 57344); codes are produced by the hardware conversion
+// cvt.rn.satfinite.{e4m3x2,e5m2x2}.f32 and widened again through f16, which holds every
+// FP8 value exactly.  PAYLOAD: 1 int8, 2 E4M3, 3 E5M2.
+template <int PAYLOAD> struct Fp8Format;
+template <> struct Fp8Format<2> { static constexpr float kMax = 448.0f, kFlush = 0x1p-117f; };
+template <> struct Fp8Format<3> { static constexpr float kMax = 57344.0f, kFlush = 0x1p-110f; };
+
+template <int PAYLOAD>
+__device__ __forceinline__ uint32_t f32x2_to_fp8x2(float lo, float hi) {
+    uint16_t d;
+    if (PAYLOAD == 2) asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(d) : "f"(hi), "f"(lo));
+    else asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
+template <int PAYLOAD>
+__device__ __forceinline__ void fp8x4_to_f32(uint32_t w, float& f0, float& f1, float& f2, float& f3) {
+    uint32_t h01, h23;
+    if (PAYLOAD == 2) {
+        asm("{\n\t.reg .b16 a, b;\n\tmov.b32 {a, b}, %2;\n\tcvt.rn.f16x2.e4m3x2 %0, a;\n\tcvt.rn.f16x2.e4m3x2 %1, b;\n\t}"
+            : "=r"(h01), "=r"(h23) : "r"(w));
+    } else {
+        asm("{\n\t.reg .b16 a, b;\n\tmov.b32 {a, b}, %2;\n\tcvt.rn.f16x2.e5m2x2 %0, a;\n\tcvt.rn.f16x2.e5m2x2 %1, b;\n\t}"
+            : "=r"(h01), "=r"(h23) : "r"(w));
+    }
+    asm("{\n\t.reg .b16 a, b;\n\tmov.b32 {a, b}, %2;\n\tcvt.f32.f16 %0, a;\n\tcvt.f32.f16 %1, b;\n\t}"
+        : "=f"(f0), "=f"(f1) : "r"(h01));
+    asm("{\n\t.reg .b16 a, b;\n\tmov.b32 {a, b}, %2;\n\tcvt.f32.f16 %0, a;\n\tcvt.f32.f16 %1, b;\n\t}"
+        : "=f"(f2), "=f"(f3) : "r"(h23));
+}
+
+// payload bytes -> fp32, exact
+template <int PAYLOAD>
+__device__ __forceinline__ void decode_x16(const uint4& c, float (&q)[16]) {
+    if (PAYLOAD == 1) {
+        codes_to_f32x16(c, q);
+    } else {
+        fp8x4_to_f32<PAYLOAD>(c.x, q[0], q[1], q[2], q[3]);
+        fp8x4_to_f32<PAYLOAD>(c.y, q[4], q[5], q[6], q[7]);
+        fp8x4_to_f32<PAYLOAD>(c.z, q[8], q[9], q[10], q[11]);
+        fp8x4_to_f32<PAYLOAD>(c.w, q[12], q[13], q[14], q[15]);
+    }
+}
+
+// the block quantizer for any payload (PAYLOAD 1 is quantize_lane)
+template <int LPB, int PAYLOAD>
+__device__ __forceinline__ void quantize_lane_payload(const float (&v)[16], uint4& codes, float& scale, float neg_zero) {
+    if (PAYLOAD == 1) {
+        quantize_lane<LPB>(v, codes, scale, neg_zero);
+        return;
+    }
+    constexpr int F = PAYLOAD == 1 ? 2 : PAYLOAD;
+    float m = max3(fabsf(v[0]), fabsf(v[1]), fabsf(v[2]));
+    float m1 = max3(fabsf(v[3]), fabsf(v[4]), fabsf(v[5]));
+    float m2 = max3(fabsf(v[6]), fabsf(v[7]), fabsf(v[8]));
+    float m3 = max3(fabsf(v[9]), fabsf(v[10]), fabsf(v[11]));
+    m = max3(m, fabsf(v[12]), fabsf(v[13]));
+    m1 = max3(m1, fabsf(v[14]), fabsf(v[15]));
+    m = max3(m, m1, fmaxf(m2, m3));
+    m = block_max<LPB>(m);
+    const bool odd = threadIdx.x & 1u;
+    const float quot = __fdiv_rn(odd ? Fp8Format<F>::kMax : m, odd ? m : Fp8Format<F>::kMax);
+    const float keep = m >= Fp8Format<F>::kFlush ? quot : 0.0f;
+    scale = __shfl_sync(0xFFFFFFFFu, keep, (threadIdx.x & 30u));
+    const float inv = __shfl_sync(0xFFFFFFFFu, keep, (threadIdx.x & 30u) | 1u);
+    uint32_t o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        float t0, t1, t2, t3;
+        mul2_rn(t0, t1, v[4 * j + 0], v[4 * j + 1], inv);
+        mul2_rn(t2, t3, v[4 * j + 2], v[4 * j + 3], inv);
+        o[j] = f32x2_to_fp8x2<F>(t0, t1) | (f32x2_to_fp8x2<F>(t2, t3) << 16);
+    }
+    codes = make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+template <int PAYLOAD>
+__device__ __forceinline__ void dequant_add_payload(const uint4& c, float scale, float (&v)[16]) {
+    float q[16];
+    decode_x16<PAYLOAD>(c, q);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) fma2_rn(v[2 * i], v[2 * i + 1], q[2 * i], q[2 * i + 1], scale, v[2 * i], v[2 * i + 1]);
+}
+
+template <int PAYLOAD>
+__device__ __forceinline__ Vec8 dequant_to_bf16_payload(const uint4& c, float scale) {
+    float q[16];
+    decode_x16<PAYLOAD>(c, q);
+    Vec8 o;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        float lo, hi;
+        mul2_rn(lo, hi, q[2 * i], q[2 * i + 1], scale);
+        o.w[i] = pack_bf16x2_rn(lo, hi);
+    }
+    return o;
+}
+
 // ---------------------------------------------------------------- message layouts
 // SPLIT   (the per-step entry points): codes[count] and scales[count/B] are separate arrays.
 // RECORDS (the simulations): a message is a sequence of 544-byte records, one per tile of
@@ -552,17 +652,17 @@ struct FlavourArgs {
 };
 
 // One hop of a chain.  Sender side: the message of v (quantized record or bf16).  Receiver side
-// (the neighbouring lane): v_out = message (+) addend; with QUANT one fused multiply-add in fp32,
+// (the neighbouring lane): v_out = message (+) addend; with a quantized payload one fused multiply-add in fp32,
 // else an fp32 add rounded to bf16 (the BF16 baseline's hop).  `sub` is the lane's position in
 // the tile and flips with every hop.
-template <int LPB, bool QUANT>
+template <int LPB, int PAYLOAD>
 __device__ __forceinline__ void chain_hop(const float (&v)[16], const float (&addend)[16], float (&v_out)[16],
                                           char* entry, char* trace_rec, uint32_t lane, uint32_t& sub, bool active,
                                           float neg_zero) {
-    if (QUANT) {
+    if (PAYLOAD != 0) {
         uint4 codes;
         float scale;
-        quantize_lane<LPB>(v, codes, scale, neg_zero);
+        quantize_lane_payload<LPB, PAYLOAD == 0 ? 1 : PAYLOAD>(v, codes, scale, neg_zero);
         const uint32_t d = (sub ^ lane) & 1u;                  // position p is held by lane p ^ d
         float hdr = __shfl_sync(0xFFFFFFFFu, scale, ((lane * LPB) & 31u) ^ d);
         if (lane >= 32u / LPB) hdr = 0.0f;
@@ -582,7 +682,7 @@ __device__ __forceinline__ void chain_hop(const float (&v)[16], const float (&ad
         }
 #pragma unroll
         for (int i = 0; i < 16; ++i) v_out[i] = addend[i];
-        dequant_add_x16(c, s, v_out);
+        dequant_add_payload<PAYLOAD == 0 ? 1 : PAYLOAD>(c, s, v_out);
     } else {
         Vec8 m;
 #pragma unroll
@@ -602,8 +702,9 @@ __device__ __forceinline__ void chain_hop(const float (&v)[16], const float (&ad
     }
 }
 
-template <int LPB, bool SEMI, bool QRS, bool QAG>
+template <int LPB, bool SEMI, bool QRS, bool QAG, int PAYLOAD>
 __global__ void __launch_bounds__(kPipeThreads) flavour_kernel(const __grid_constant__ FlavourArgs a) {
+    constexpr int RS = QRS ? PAYLOAD : 0;          // payload of the reduce-scatter hops (0: bf16 messages)
     const uint32_t lane = threadIdx.x & 31u;
     const uint64_t warps = (uint64_t)gridDim.x * (kPipeThreads / 32);
     const uint64_t warp = (uint64_t)blockIdx.x * (kPipeThreads / 32) + (threadIdx.x >> 5);
@@ -638,7 +739,7 @@ __global__ void __launch_bounds__(kPipeThreads) flavour_kernel(const __grid_cons
             for (uint32_t j = 1; j < N; ++j) {                                   // hop into rank k+1+j
                 float x[16];
                 load_shard(k + 1 + j, sub ^ 1u, x);
-                chain_hop<LPB, QRS>(acc, x, acc, fifo + (hops & 1u) * kFifoEntryBytes, QRS ? trace_of(j - 1) : nullptr,
+                chain_hop<LPB, RS>(acc, x, acc, fifo + (hops & 1u) * kFifoEntryBytes, QRS ? trace_of(j - 1) : nullptr,
                                     lane, sub, active, a.neg_zero);
                 ++hops;
             }
@@ -656,9 +757,9 @@ __global__ void __launch_bounds__(kPipeThreads) flavour_kernel(const __grid_cons
                     if (j + 1 < h) {
                         float x[16];
                         load_shard(k + h + 1 + j, sub ^ 1u, x);
-                        chain_hop<LPB, QRS>(v, x, v, entry, tr, lane, sub, active, a.neg_zero);
+                        chain_hop<LPB, RS>(v, x, v, entry, tr, lane, sub, active, a.neg_zero);
                     } else {
-                        chain_hop<LPB, QRS>(v, acc, acc, entry, tr, lane, sub, active, a.neg_zero);
+                        chain_hop<LPB, RS>(v, acc, acc, entry, tr, lane, sub, active, a.neg_zero);
                     }
                     ++hops;
                 }
@@ -673,9 +774,9 @@ __global__ void __launch_bounds__(kPipeThreads) flavour_kernel(const __grid_cons
                 if (j < h) {
                     float x[16];
                     load_shard(k + h - j, sub ^ 1u, x);
-                    chain_hop<LPB, QRS>(v, x, v, entry, tr, lane, sub, active, a.neg_zero);
+                    chain_hop<LPB, RS>(v, x, v, entry, tr, lane, sub, active, a.neg_zero);
                 } else {
-                    chain_hop<LPB, QRS>(v, acc, acc, entry, tr, lane, sub, active, a.neg_zero);
+                    chain_hop<LPB, RS>(v, acc, acc, entry, tr, lane, sub, active, a.neg_zero);
                 }
                 ++hops;
             }
@@ -688,7 +789,7 @@ __global__ void __launch_bounds__(kPipeThreads) flavour_kernel(const __grid_cons
             if (QAG) {
                 uint4 codes;
                 float scale;
-                quantize_lane<LPB>(acc, codes, scale, a.neg_zero);
+                quantize_lane_payload<LPB, PAYLOAD>(acc, codes, scale, a.neg_zero);
                 const uint32_t d = (sub ^ lane) & 1u;
                 float hdr = __shfl_sync(0xFFFFFFFFu, scale, ((lane * LPB) & 31u) ^ d);
                 if (lane >= 32u / LPB) hdr = 0.0f;
@@ -707,7 +808,7 @@ __global__ void __launch_bounds__(kPipeThreads) flavour_kernel(const __grid_cons
                     c = ld_coherent_128(entry + kRecordHeader + sub * 16);
                     s = ld_coherent_f32(reinterpret_cast<const float*>(entry) + sub / LPB);
                 }
-                o = dequant_to_bf16x16(c, s);
+                o = dequant_to_bf16_payload<PAYLOAD>(c, s);
             } else {
                 Vec8 m;
 #pragma unroll

@@ -63,6 +63,26 @@ def f32_word(q: Fraction) -> int:
     return u
 
 
+# FP8 formats: significand bits, minimum exponent, largest finite value, flush threshold
+FP8 = {"e4m3": dict(p=4, emin=-6, fmax=Fraction(448), flush=Fraction(2) ** -117),
+       "e5m2": dict(p=3, emin=-14, fmax=Fraction(57344), flush=Fraction(2) ** -110)}
+
+
+def quantize_block_fp8(v, fmt):
+    """v: Fractions that are fp32 values -> (scale, code VALUES as Fractions)."""
+    f = FP8[fmt]
+    amax = max(abs(t) for t in v)
+    if amax < f["flush"]:
+        return Fraction(0), [Fraction(0)] * len(v)
+    scale = f32(amax / f["fmax"])
+    inv = f32(f["fmax"] / amax)
+    vals = []
+    for t in v:
+        r = round_to(f32(t * inv), f["p"], f["emin"])
+        vals.append(max(-f["fmax"], min(f["fmax"], r)))
+    return scale, vals
+
+
 def quantize_block(v):
     """v: list of Fractions that are fp32 values -> (scale Fraction, codes list[int])."""
     amax = max(abs(t) for t in v)
@@ -74,7 +94,7 @@ def quantize_block(v):
     return scale, codes
 
 
-def chain_allreduce(words, block):
+def chain_allreduce(words, block, payload="int8"):
     """words[r][i]: bf16 words, N ranks x count.  Per-shard adder chains.
 
     Shard k is reduced along ranks k+1, k+2, ..., k (mod N); every link
@@ -92,7 +112,7 @@ def chain_allreduce(words, block):
             order = [(k + 1 + j) % n_ranks for j in range(n_ranks)]
             v = [frac_from_bf16_word(words[order[0]][i]) for i in idx]
             for j in range(n_ranks):
-                scale, codes = quantize_block(v)
+                scale, codes = quantize_block(v) if payload == "int8" else quantize_block_fp8(v, payload)
                 events[(k, b, j)] = (scale, codes)
                 if j < n_ranks - 1:
                     nxt = order[j + 1]

@@ -23,6 +23,10 @@ def decode(flavour):
     return bool(flavour & eq.FLAVOUR_SEMI_LOOP), bool(flavour & eq.FLAVOUR_QUANT_RS), bool(flavour & eq.FLAVOUR_QUANT_AG)
 
 
+def payload_of(flavour):
+    return "e4m3" if flavour & eq.FLAVOUR_E4M3 else "e5m2" if flavour & eq.FLAVOUR_E5M2 else "int8"
+
+
 def run_flavour(gu, xd, block, flavour, keep_trace):
     n, count = xd.shape
     wb = eq.allreduce_sim_flavour_workspace_bytes(n, count, block, flavour, keep_trace)
@@ -41,7 +45,7 @@ def run_flavour(gu, xd, block, flavour, keep_trace):
 def compare(gu, x, block, flavour):
     semi, qr, qa = decode(flavour)
     n, count = x.shape
-    res = oracle.allreduce_variant(wl.as_u16(x), block, semi, qr, qa, trace=True)
+    res = oracle.allreduce_variant(wl.as_u16(x), block, semi, qr, qa, trace=True, payload=payload_of(flavour))
     out, ws = run_flavour(gu, x.cuda(), block, flavour, True)
     gu.assert_same_words(out, res["out"], f"flavour {flavour} outputs")
     sc, co = eq.trace_views(ws.u8[binding.FLAVOUR_FIFO_BYTES:], n, count, block, keep_trace=True)
@@ -109,10 +113,44 @@ def test_flavour_argument_errors(gu):
     ws = torch.empty(binding.FLAVOUR_FIFO_BYTES, dtype=torch.uint8, device="cuda")
     args = ([x[r] for r in range(3)], [out[r] for r in range(3)], 3, 3 * 64, 64)
     with pytest.raises(eq.EquarxError) as e:
-        eq.allreduce_sim_flavour(*args, 8, ws, ws.numel())
+        eq.allreduce_sim_flavour(*args, 32, ws, ws.numel())
     assert e.value.status == binding.ERR_FLAVOUR
     with pytest.raises(eq.EquarxError) as e:
         eq.allreduce_sim_flavour(*args, eq.FLAVOUR_SEMI_LOOP, ws, ws.numel())      # odd rank count
     assert e.value.status == binding.ERR_NRANKS
     assert eq.allreduce_sim_flavour_workspace_bytes(3, 3 * 64, 64, 1) == 0
     assert eq.allreduce_sim_flavour_workspace_bytes(4, 4 * 64, 64, 1) == binding.FLAVOUR_FIFO_BYTES
+
+
+FP8_FLAVOURS = [sched | fmt for fmt in (eq.FLAVOUR_E4M3, eq.FLAVOUR_E5M2) for sched in (2, 3, 4, 5, 6, 7)]
+
+
+@pytest.mark.parametrize("flavour", FP8_FLAVOURS)
+@pytest.mark.parametrize("nranks,block", [(2, 64), (4, 512), (8, 256), (16, 128)])
+def test_fp8_flavours_match_oracle(gu, flavour, nranks, block):
+    bps = 5 if block >= 256 else 19
+    w = wl.Workload("t", nranks, nranks * bps * block, block, "normal", seed=nranks + flavour)
+    compare(gu, wl.make_inputs(w), block, flavour)
+
+
+@pytest.mark.parametrize("flavour", (6 | eq.FLAVOUR_E4M3, 6 | eq.FLAVOUR_E5M2, 7 | eq.FLAVOUR_E4M3))
+@pytest.mark.parametrize("kind", ("wide", "tiny", "huge", "halves", "zeros"))
+def test_fp8_value_ranges(gu, flavour, kind):
+    """40-binade data, data around the flush thresholds and FP8 subnormals, near the bf16 maximum,
+    exact ties, signed zeros."""
+    from test_gpu_parity import _values
+    n, block = 4, 128
+    x = torch.stack([_values(kind, n * block * 7, 50 + r) for r in range(n)])
+    compare(gu, x, block, flavour)
+
+
+@pytest.mark.parametrize("flavour", (6 | eq.FLAVOUR_E4M3, 6 | eq.FLAVOUR_E5M2))
+def test_fp8_stress_blocks(gu, flavour):
+    compare(gu, wl.make_inputs(wl.C5, count=64 * 256 * 4), 256, flavour)
+
+
+def test_fp8_flavour_bits_are_validated(gu):
+    assert eq.allreduce_sim_flavour_workspace_bytes(4, 4 * 64, 64, eq.FLAVOUR_E4M3) == 0            # nothing quantized
+    assert eq.allreduce_sim_flavour_workspace_bytes(4, 4 * 64, 64, 6 | eq.FLAVOUR_E4M3 | eq.FLAVOUR_E5M2) == 0
+    assert eq.allreduce_sim_flavour_workspace_bytes(4, 4 * 64, 64, 6 | eq.FLAVOUR_E5M2) == binding.FLAVOUR_FIFO_BYTES
+    assert eq.allreduce_sim_flavour_workspace_bytes(4, 4 * 64, 64, 32) == 0

@@ -147,3 +147,74 @@ def test_variant_argument_errors():
     x = np.zeros((3, 3 * 64), np.uint16)
     with pytest.raises(oracle.OracleError):
         oracle.allreduce_variant(x, 64, semi_loop=True)        # odd number of ranks
+
+
+# ---------------------------------------------------------------- FP8 payloads
+from conftest import load_golden            # noqa: E402
+from exact_fp import chain_allreduce         # noqa: E402
+
+FP8_GOLD = load_golden("hand_blocks_fp8.txt")
+
+
+@pytest.mark.parametrize("fmt", ["e4m3", "e5m2"])
+def test_fp8_hand_worked_block(fmt):
+    g = FP8_GOLD[fmt]
+    x = words_of([float(v) for v in g["x"]])[None, :]
+    res = oracle.allreduce_variant(x, 8, False, True, True, trace=True, payload=fmt)
+    assert res["scales"][0, 0, 0].view(np.uint32) == int(g["scale"][0], 16)
+    assert [int(c) & 0xFF for c in res["codes"][0, 0]] == [int(c, 16) for c in g["codes"]]
+    assert np.array_equal(to_f64(res["out"][0]), np.array([float(v) for v in g["out"]]))
+
+
+def _fp8_value(byte, fmt):
+    p, emin, bias = (4, -6, 7) if fmt == "e4m3" else (3, -14, 15)
+    field, mant = (byte & 0x7F) >> (p - 1), byte & ((1 << (p - 1)) - 1)
+    a = mant * 2.0 ** (emin - (p - 1)) if field == 0 else (1 + mant / 2 ** (p - 1)) * 2.0 ** (field - bias)
+    return -a if byte & 0x80 else a
+
+
+@pytest.mark.parametrize("fmt", ["e4m3", "e5m2"])
+@pytest.mark.parametrize("kind", ["normal", "wide", "tiny"])
+@pytest.mark.parametrize("nranks,block,bps", [(1, 4, 2), (2, 3, 1), (3, 5, 2), (4, 8, 1)])
+def test_fp8_brute_force_exact_rational(fmt, kind, nranks, block, bps):
+    from test_oracle_pins_chain import rand_bf16
+    from exact_fp import f32_word
+    rng = np.random.default_rng(hash((fmt, kind, nranks, block)) % (2 ** 32))
+    x = rand_bf16(rng, (nranks, nranks * block * bps), kind)
+    res = oracle.allreduce_variant(x, block, False, True, True, trace=True, payload=fmt)
+    out, events = chain_allreduce([[int(w) for w in row] for row in x], block, payload=fmt)
+    for r in range(nranks):
+        # FP8 has a negative zero code and the rational model has no signed zero: compare -0 as 0
+        assert [0 if int(w) == 0x8000 else int(w) for w in res["out"][r]] == out
+    for (k, b, j), (scale, vals) in events.items():
+        assert int(res["scales"][k, j, b].view(np.uint32)) == f32_word(scale)
+        got = [_fp8_value(int(c) & 0xFF, fmt) for c in res["codes"][k, j, b * block:(b + 1) * block]]
+        assert got == [float(v) for v in vals]
+
+
+@pytest.mark.parametrize("fmt,top", [("e4m3", 448.0), ("e5m2", 57344.0)])
+def test_fp8_invariants(fmt, top):
+    """Every non-zero event has a code of magnitude FMAX; outputs identical on all ranks;
+    scaling all inputs by a power of two scales scales and outputs and leaves the codes alone."""
+    x = wl.as_u16(wl.make_inputs(wl.Workload("t", 4, 4 * 64 * 6, 64, "normal", seed=3)))
+    res = oracle.allreduce_variant(x, 64, False, True, True, trace=True, payload=fmt)
+    vals = np.vectorize(lambda c: _fp8_value(int(c) & 0xFF, fmt))(res["codes"]).reshape(4, 4, -1, 64)
+    assert np.all(np.abs(vals).max(axis=3) == top)
+    for r in range(1, 4):
+        assert np.array_equal(res["out"][0], res["out"][r])
+    y = torch.tensor(to_f64(x) * 2.0 ** 7).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    res2 = oracle.allreduce_variant(y, 64, False, True, True, trace=True, payload=fmt)
+    assert np.array_equal(res2["codes"], res["codes"])
+    assert np.array_equal(res2["scales"], res["scales"] * np.float32(128.0))
+    assert np.array_equal(to_f64(res2["out"]), to_f64(res["out"]) * 128.0)
+
+
+def test_fp8_error_is_larger_than_int8_and_ordered():
+    """With 3 and 2 mantissa bits the FP8 payloads are coarser than int8 on N(0,1) data."""
+    x = wl.as_u16(wl.make_inputs(wl.Workload("t", 8, 8 * 64 * 256, 64, "normal", seed=0)))
+    exact = to_f64(x).sum(axis=0)
+    mse = {}
+    for fmt in ("int8", "e4m3", "e5m2"):
+        d = to_f64(oracle.allreduce_variant(x, 64, False, True, True, payload=fmt)["out"][0]) - exact
+        mse[fmt] = float(np.mean(d * d))
+    assert mse["int8"] < mse["e4m3"] < mse["e5m2"]
