@@ -345,10 +345,14 @@ int equarx_allreduce_sim_pipelined(const void* const* in_bf16, void* const* out_
 
     const void* kernel = nullptr;
     switch (block) {
-        case 64: kernel = reinterpret_cast<const void*>(pipelined_kernel<4>); break;
-        case 128: kernel = reinterpret_cast<const void*>(pipelined_kernel<8>); break;
-        case 256: kernel = reinterpret_cast<const void*>(pipelined_kernel<16>); break;
-        default: kernel = reinterpret_cast<const void*>(pipelined_kernel<32>); break;
+        case 64: kernel = keep_trace ? reinterpret_cast<const void*>(pipelined_kernel<4, true>)
+                                     : reinterpret_cast<const void*>(pipelined_kernel<4, false>); break;
+        case 128: kernel = keep_trace ? reinterpret_cast<const void*>(pipelined_kernel<8, true>)
+                                      : reinterpret_cast<const void*>(pipelined_kernel<8, false>); break;
+        case 256: kernel = keep_trace ? reinterpret_cast<const void*>(pipelined_kernel<16, true>)
+                                      : reinterpret_cast<const void*>(pipelined_kernel<16, false>); break;
+        default: kernel = keep_trace ? reinterpret_cast<const void*>(pipelined_kernel<32, true>)
+                                     : reinterpret_cast<const void*>(pipelined_kernel<32, false>); break;
     }
     // persistent grid: a whole number of CTAs per SM
     int dev = 0, sms = 0, occ = 0;

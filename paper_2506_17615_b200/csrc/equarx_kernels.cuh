@@ -547,10 +547,10 @@ __global__ void __launch_bounds__(kThreads) ag_dequant_kernel(const __grid_const
 // The bf16 shard of the next step is prefetched while a step computes.
 constexpr int kPipeThreads = 64;
 #ifndef EQX_PIPE_MINBLOCKS
-#define EQX_PIPE_MINBLOCKS 16
+#define EQX_PIPE_MINBLOCKS 18
 #endif
 
-template <int LPB>
+template <int LPB, bool TRACE>
 __global__ void __launch_bounds__(kPipeThreads, EQX_PIPE_MINBLOCKS) pipelined_kernel(const __grid_constant__ PipeArgs a) {
     const uint32_t lane = threadIdx.x & 31u;
     const uint64_t warps = (uint64_t)gridDim.x * (kPipeThreads / 32);
@@ -558,75 +558,102 @@ __global__ void __launch_bounds__(kPipeThreads, EQX_PIPE_MINBLOCKS) pipelined_ke
     const uint32_t N = a.nranks;
     const uint64_t groups = a.shard >> 4;
     const uint64_t tiles = a.tiles_per_shard * N;
+    const uint64_t trace_stride = a.tiles_per_shard * kRecordBytes;      // one event further in the trace
     char* const fifo = a.records + warp * (2 * kRecordBytes);
+    // byte offsets inside a record: even steps send from position `lane` and receive (as the
+    // neighbouring lane, acting for the receiving rank) at position lane ^ 1; odd steps the reverse
+    const uint32_t code_own = kRecordHeader + lane * 16, code_nbr = kRecordHeader + (lane ^ 1u) * 16;
+    const uint32_t scale_own = (lane / LPB) * 4, scale_nbr = ((lane ^ 1u) / LPB) * 4;
+    const uint32_t hdr_src_even = (lane * LPB) & 31u, hdr_src_odd = hdr_src_even ^ 1u;
 
-    // the first shard of a tile is fetched while the previous tile finishes (its last step needs
-    // no prefetch of its own, so the same registers are free)
-    auto first_shard = [&](uint64_t tile_) {
-        Vec8 x = {};
-        if (tile_ < tiles) {
-            const uint32_t k_ = (uint32_t)(tile_ / a.tiles_per_shard);
-            const uint64_t t_ = tile_ - (uint64_t)k_ * a.tiles_per_shard;
-            const uint32_t rho_ = k_ + 1 == N ? 0 : k_ + 1;
-            if (t_ * 32 + lane < groups)
-                x = ld_coherent_256(static_cast<const char*>(a.in[rho_]) + ((uint64_t)k_ * a.shard + (t_ * 32 + lane) * 16) * 2);
-        }
-        return x;
+    // byte offset of this lane's own group of a tile in every rank's tensor (the neighbouring group
+    // is 32 bytes to the other side); ~0 if the lane is past the end of a ragged last tile
+    auto own_offset = [&](uint64_t tile_, uint32_t& k_) -> uint64_t {
+        k_ = (uint32_t)(tile_ / a.tiles_per_shard);
+        const uint64_t t_ = tile_ - (uint64_t)k_ * a.tiles_per_shard;
+        if (t_ * 32 + lane >= groups) return ~uint64_t(0);
+        return ((uint64_t)k_ * a.shard + (t_ * 32 + lane) * 16) * 2;
     };
-    Vec8 xw = first_shard(warp);
+    // the first shard of a tile is fetched while the previous tile finishes (the last step needs
+    // no prefetch of its own, so the same registers are free)
+    uint32_t k_next = 0;
+    uint64_t off_next = warp < tiles ? own_offset(warp, k_next) : ~uint64_t(0);
+    Vec8 xw = {};
+    if (off_next != ~uint64_t(0))
+        xw = ld_coherent_256(static_cast<const char*>(a.in[k_next + 1 == N ? 0 : k_next + 1]) + off_next);
 
     for (uint64_t tile = warp; tile < tiles; tile += warps) {
-        const uint32_t k = (uint32_t)(tile / a.tiles_per_shard);           // shard
-        const uint64_t t = tile - (uint64_t)k * a.tiles_per_shard;
-        const uint64_t g = t * 32 + lane;              // this lane's group at even steps; g ^ 1 at odd steps
-        const bool active = g < groups;                // groups is a multiple of 4: lane pairs are in or out together
-        const uint64_t shard_off = (uint64_t)k * a.shard;
-        char* const trace = a.records + ((uint64_t)k * N * a.tiles_per_shard + t) * kRecordBytes;
-
+        const uint32_t k = k_next;
+        const uint64_t off_own = off_next;
+        const bool active = off_own != ~uint64_t(0);   // lane pairs are in or out together (groups % 4 == 0)
+        const uint64_t off_nbr = off_own ^ 32;         // the neighbouring lane's group
+        char* trace = TRACE ? a.records + ((uint64_t)k * N * a.tiles_per_shard + (tile - (uint64_t)k * a.tiles_per_shard)) * kRecordBytes
+                            : nullptr;
         uint32_t rho = k + 1 == N ? 0 : k + 1;         // rank of step 0
         float v[16];
         widen_bf16x16(xw, v);
-        uint32_t sub = lane;                           // position inside the tile handled at step j
-        for (uint32_t j = 0;; ++j) {
+
+        // next shard (or, at the last step, the first shard of this warp's next tile)
+        auto prefetch = [&](uint32_t j, uint64_t off) {
             rho = rho + 1 == N ? 0 : rho + 1;
-            if (j + 1 < N) {                           // the next step's bf16 shard arrives while this step computes
-                if (active)
-                    xw = ld_coherent_256(static_cast<const char*>(a.in[rho]) + (shard_off + (t * 32 + (sub ^ 1)) * 16) * 2);
+            if (j + 1 < N) {
+                if (active) xw = ld_coherent_256(static_cast<const char*>(a.in[rho]) + off);
             } else {
-                xw = first_shard(tile + warps);        // last step: fetch the next tile's first shard instead
+                xw = Vec8{};
+                off_next = tile + warps < tiles ? own_offset(tile + warps, k_next) : ~uint64_t(0);
+                if (off_next != ~uint64_t(0))
+                    xw = ld_coherent_256(static_cast<const char*>(a.in[k_next + 1 == N ? 0 : k_next + 1]) + off_next);
             }
+        };
+        // one ring step: quantize v, send the record, receive it as the neighbouring lane
+        auto exchange = [&](char* rec, uint32_t hdr_src, uint32_t code_send, uint32_t code_recv, uint32_t scale_recv,
+                            uint4& c, float& s) {
             uint4 codes;
             float scale;
             quantize_lane<LPB>(v, codes, scale, a.neg_zero);
-            char* const rec = a.keep_trace ? trace + (uint64_t)j * a.tiles_per_shard * kRecordBytes
-                                           : fifo + (j & 1u) * kRecordBytes;
-            // the sender's view: position `sub` of the tile
-            {
-                float hdr = __shfl_sync(0xFFFFFFFFu, scale, ((lane * LPB) & 31u) ^ (j & 1u));
-                if (lane >= 32u / LPB) hdr = 0.0f;
-                if (lane < 8 && t * 32 < groups) st_plain_f32(reinterpret_cast<float*>(rec) + lane, hdr);
-                if (active) st_plain_128(rec + kRecordHeader + sub * 16, codes);
-            }
-            __syncwarp();                              // the message is now visible to the neighbouring lane,
-            sub ^= 1;                                  // which acts for the receiving rank on the neighbour's group
-            uint4 c = make_uint4(0, 0, 0, 0);
-            float s = 0.0f;
+            float hdr = __shfl_sync(0xFFFFFFFFu, scale, hdr_src);       // lanes 0..7 write the metadata sector
+            if (lane >= 32u / LPB) hdr = 0.0f;
+            if (lane < 8) st_plain_f32(reinterpret_cast<float*>(rec) + lane, hdr);
+            if (active) st_plain_128(rec + code_send, codes);
+            __syncwarp();                              // the message is now visible to the neighbouring lane
+            c = make_uint4(0, 0, 0, 0);
+            s = 0.0f;
             if (active) {
-                c = ld_coherent_128(rec + kRecordHeader + sub * 16);
-                s = ld_coherent_f32(reinterpret_cast<const float*>(rec) + sub / LPB);
+                c = ld_coherent_128(rec + code_recv);
+                s = ld_coherent_f32(reinterpret_cast<const float*>(rec + scale_recv));
             }
-            if (j + 1 == N) {                          // all-gather: dequantize to bf16, one store per rank
-                const Vec8 o = dequant_to_bf16x16(c, s);
-                if (active) {
-                    const uint64_t byte_off = (shard_off + (t * 32 + sub) * 16) * 2;
-                    for (uint32_t r = 0; r < N; ++r) st_stream_256(static_cast<char*>(a.out[r]) + byte_off, o);
-                }
+            // a FIFO entry is overwritten two steps later, after the __syncwarp of the step in between:
+            // every lane's load above has returned by then, because its value feeds that step's quantization
+        };
+        auto gather = [&](const uint4& c, float s, uint64_t off) {      // all-gather: one store per rank
+            const Vec8 o = dequant_to_bf16x16(c, s);
+            if (active)
+                for (uint32_t r = 0; r < N; ++r) st_stream_256(static_cast<char*>(a.out[r]) + off, o);
+        };
+
+        for (uint32_t j = 0;; j += 2) {
+            uint4 c;
+            float s;
+            // even step: send from the own position, receive at the neighbour's
+            prefetch(j, off_nbr);
+            exchange(TRACE ? trace : fifo, hdr_src_even, code_own, code_nbr, scale_nbr, c, s);
+            if (j + 1 == N) {
+                gather(c, s, off_nbr);
                 break;
             }
             widen_bf16x16(xw, v);
             dequant_add_x16(c, s, v);
-            // FIFO entry (j & 1) is overwritten at step j+2, after the __syncwarp of step j+1: every
-            // lane's load above has returned by then, because its value feeds the quantization of step j+1
+            if (TRACE) trace += trace_stride;
+            // odd step: send from the neighbour's position, receive at the own
+            prefetch(j + 1, off_own);
+            exchange(TRACE ? trace : fifo + kRecordBytes, hdr_src_odd, code_nbr, code_own, scale_own, c, s);
+            if (j + 2 == N) {
+                gather(c, s, off_own);
+                break;
+            }
+            widen_bf16x16(xw, v);
+            dequant_add_x16(c, s, v);
+            if (TRACE) trace += trace_stride;
         }
         __syncwarp();                                  // the next tile reuses the FIFO
     }
