@@ -211,6 +211,8 @@ def max_over_ranks(ms, world, device):
         return ms
     import torch
     import torch.distributed as dist
+    if dist.get_backend() == "gloo":
+        device = torch.device("cpu")
     t = torch.tensor([ms], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
@@ -251,7 +253,14 @@ def main():
     if world > 1:
         import torch.distributed as dist
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=dev)
+        try:
+            dist.init_process_group("nccl", device_id=dev)
+            dist.barrier()
+        except Exception as exc:      # the data path has no collective: any backend can carry the barrier
+            print(f"bench: NCCL unavailable ({exc!r}); using gloo for the barrier and the max", file=sys.stderr)
+            if dist.is_initialized():
+                dist.destroy_process_group()
+            dist.init_process_group("gloo")
 
     def barrier():
         if world > 1:

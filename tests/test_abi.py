@@ -161,3 +161,24 @@ def test_bf16_sim_rejects_bad_arguments():
 
 def test_no_cuda_error_recorded_by_validation():
     assert eq.last_cuda_error() == 0
+
+
+def test_rounded_code_never_leaves_the_int8_range_without_a_clamp():
+    """The kernels omit the oracle's clamp to [-127, 127].  That is safe iff
+    rne(fl(amax * fl(127 / amax))) == 127 for every block maximum: the largest |v| of a block
+    gives the largest product, and multiplication by a positive constant is monotone.  Checked
+    for every fp32 mantissa in several binades (scaling amax by a power of two scales
+    fl(127 / amax) by the inverse power exactly, as long as nothing leaves the normal range),
+    including the smallest block that is still quantized (2^-118) and the bf16 maximum."""
+    import numpy as np
+    mant = np.arange(1 << 23, dtype=np.uint32)
+    for exp_field in (9, 64, 127, 128, 200, 254):          # 2^-118, ..., 1, 2, ..., up to 2^127
+        amax = ((np.uint32(exp_field) << np.uint32(23)) | mant).view(np.float32)
+        inv = np.float32(127.0) / amax
+        assert np.all(np.isfinite(inv)) and np.all(inv > 0)
+        top = amax * inv                                   # fp32 multiply, round to nearest even
+        assert top.dtype == np.float32
+        assert float(top.max()) < 127.5 and float(top.min()) > 126.5
+        # and the scale that travels is a normal number
+        scale = amax / np.float32(127.0)
+        assert float(scale.min()) >= 2.0 ** -126
