@@ -23,8 +23,9 @@
  *   - `block` is the number of contiguous elements that share one fp32
  *     scale (Section 3.2, Fig. 3: one scale factor per block of entries);
  *     supported values 64, 128, 256, 512.
- *   - Inputs must be finite.  Inf/NaN are outside the contract: no trap,
- *     result unspecified.
+ *   - Inputs must be finite, and so must every fp32 partial sum along a
+ *     chain (|sum| below the fp32 maximum).  Inf/NaN inputs and overflowing
+ *     sums are outside the contract: no trap, result unspecified.
  *
  * Arithmetic (identical, bit for bit, in every entry point)
  *   amax  = max |v| over the block                      (Section 3.2, max reduction)

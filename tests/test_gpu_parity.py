@@ -15,7 +15,7 @@ pytestmark = pytest.mark.gpu
 BLOCKS = (64, 128, 256, 512)
 
 
-def _values(kind, count, seed):
+def _values(kind, count, seed, nranks=4):
     g = torch.Generator().manual_seed(seed)
     if kind == "normal":
         v = torch.randn(count, generator=g)
@@ -27,8 +27,8 @@ def _values(kind, count, seed):
     elif kind == "tiny":        # around the flush threshold and among bf16 subnormals
         v = (torch.randint(-127, 128, (count,), generator=g).double()
              * torch.exp2(torch.randint(-133, -112, (count,), generator=g).double()))
-    elif kind == "huge":        # close to the bf16 maximum
-        v = torch.randn(count, generator=g).double() * 2.0 ** 125
+    elif kind == "huge":        # as large as the fp32 partial sums of nranks tensors allow (finite sums are the contract)
+        v = torch.randn(count, generator=g).clamp(-6, 6).double() * 2.0 ** 125 / (2 * max(nranks, 3))
     elif kind == "zeros":
         v = torch.zeros(count)
         v[1::7] = -0.0
@@ -281,3 +281,24 @@ def test_host_pipeline_matches_device_path(gu):
     for i in range(5):
         exp = oracle.allreduce(wl.as_u16(xs[i]), 256)["out"]
         gu.assert_same_words(h_out[i], exp, f"submission {i}")
+
+
+def _random_cases(n, seed):
+    rng = np.random.default_rng(seed)
+    cases = []
+    for _ in range(n):
+        nranks = int(rng.choice([1, 2, 3, 4, 6, 7, 8, 12, 16, 24, 32, 48, 64]))
+        block = int(rng.choice(BLOCKS))
+        bps = int(rng.integers(1, 40))
+        kind = str(rng.choice(KINDS))
+        cases.append((nranks, block, bps, kind, int(rng.integers(0, 1 << 30))))
+    return cases
+
+
+@pytest.mark.parametrize("nranks,block,bps,kind,seed", _random_cases(40, 2024))
+def test_randomized_shapes_and_value_ranges(gu, nranks, block, bps, kind, seed):
+    """Seeded random draws over rank counts, block sizes, shard lengths (ragged against the
+    512-element tile and the 4096-element CTA) and value ranges: both schedules, full trace."""
+    count = nranks * bps * block
+    x = torch.stack([_values(kind, count, seed + r, nranks) for r in range(nranks)])
+    _compare_full(gu, x, block)
