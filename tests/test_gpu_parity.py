@@ -302,3 +302,25 @@ def test_randomized_shapes_and_value_ranges(gu, nranks, block, bps, kind, seed):
     count = nranks * bps * block
     x = torch.stack([_values(kind, count, seed + r, nranks) for r in range(nranks)])
     _compare_full(gu, x, block)
+
+
+def test_pipelined_fifo_holds_the_last_messages_of_each_warp(gu):
+    """Without a trace the pipelined schedule sends every hop message through a two-record staging
+    FIFO per warp.  With at most one tile per warp, warp w's FIFO must hold, on return, the last
+    two messages (events N-2 and N-1) of tile w, as 544-byte records: metadata sector, then codes."""
+    n, block, bps = 4, 128, 8                      # shard = 1024 elements = 2 tiles; 8 tiles in all
+    count = n * bps * block
+    x = wl.make_inputs(wl.Workload("t", n, count, block, "normal", seed=77))
+    res = oracle.allreduce(wl.as_u16(x), block, trace=True)
+    _, ws = gu.run_sim(x.cuda(), block, keep_trace=False, variant="pipelined")
+    fifo = ws.u8.cpu().numpy()
+    shard, per_tile = count // n, 512 // block
+    for tile in range(n * 2):
+        k, t = divmod(tile, 2)
+        for j in (n - 2, n - 1):
+            rec = fifo[tile * 1088 + (j & 1) * 544: tile * 1088 + (j & 1) * 544 + 544]
+            hdr = rec[:32].view(np.float32)
+            exp_sc = res["scales"][k, j, t * per_tile:(t + 1) * per_tile]
+            assert np.array_equal(hdr[:per_tile].view(np.uint32), exp_sc.view(np.uint32)), (tile, j)
+            assert not hdr[per_tile:].any()
+            assert np.array_equal(rec[32:].view(np.int8), res["codes"][k, j, t * 512:(t + 1) * 512]), (tile, j)
