@@ -324,3 +324,24 @@ def test_pipelined_fifo_holds_the_last_messages_of_each_warp(gu):
             assert np.array_equal(hdr[:per_tile].view(np.uint32), exp_sc.view(np.uint32)), (tile, j)
             assert not hdr[per_tile:].any()
             assert np.array_equal(rec[32:].view(np.int8), res["codes"][k, j, t * 512:(t + 1) * 512]), (tile, j)
+
+
+@pytest.mark.parametrize("nranks", (4, 8, 16))
+@pytest.mark.parametrize("block", (128, 256, 512))
+@pytest.mark.parametrize("dist", ("uniform", "normal"))
+def test_every_sweep_point_sampled(gu, nranks, block, dist):
+    """All 15 message sizes (16 KB .. 256 MB per rank) of one (N, block, distribution) line of the
+    sweep, in the configuration the sweep times (no trace): sampled blocks of the pipelined schedule
+    against the oracle, and the launch-per-step schedule against the pipelined one, word for word."""
+    for p in range(14, 29):
+        w = wl.sweep_point(nranks, 1 << p, block, dist)
+        bps = w.count // nranks // block
+        x = wl.make_inputs(w, device="cuda")
+        out, _ = gu.run_sim(x, block, variant="pipelined")
+        picks = gu.sample_blocks(nranks, bps, 6, seed=p)
+        exp = gu.oracle_out_on_samples(x, picks, block)
+        gu.assert_same_words(gu.gather_blocks(out, picks, block), exp, w.name)
+        out2, _ = gu.run_sim(x, block, variant="steps")
+        assert torch.equal(out.view(torch.int16), out2.view(torch.int16)), w.name
+        del out, out2, x
+        torch.cuda.empty_cache()
