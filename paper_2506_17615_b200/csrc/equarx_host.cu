@@ -383,8 +383,19 @@ int equarx_allreduce_sim_pipelined(const void* const* in_bf16, void* const* out_
     const uint64_t fifo_ctas = uint64_t(EQUARX_PIPELINE_FIFO_BYTES) / (2 * kRecordBytes) / wpc;
     if (!keep_trace && best_ctas > fifo_ctas) best_ctas = fifo_ctas;
 
+    // programmatic dependent launch hides the launch latency behind the previous kernel's tail; the
+    // kernel itself waits for that kernel to complete before its first memory access
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(unsigned(best_ctas));
+    cfg.blockDim = dim3(kPipeThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = use_pdl() ? 1 : 0;
     void* params[1] = {&a};
-    e = cudaLaunchKernel(kernel, dim3(unsigned(best_ctas)), dim3(kPipeThreads), params, 0, stream);
+    e = cudaLaunchKernelExC(&cfg, kernel, params);
     if (e != cudaSuccess) {
         g_last_cuda_error = int(e);
         (void)cudaGetLastError();

@@ -566,6 +566,11 @@ __global__ void __launch_bounds__(kPipeThreads, EQX_PIPE_MINBLOCKS) pipelined_ke
     const uint32_t scale_own = (lane / LPB) * 4, scale_nbr = ((lane ^ 1u) / LPB) * 4;
     const uint32_t hdr_src_even = (lane * LPB) & 31u, hdr_src_odd = hdr_src_even ^ 1u;
 
+    // Launched as a programmatic dependent: the grid may be scheduled while the previous kernel of
+    // the stream drains, but touches no memory before that kernel has completed and flushed.
+    pdl_launch_dependents();
+    pdl_wait_prior_grid();
+
     // byte offset of this lane's own group of a tile in every rank's tensor (the neighbouring group
     // is 32 bytes to the other side); ~0 if the lane is past the end of a ragged last tile
     auto own_offset = [&](uint64_t tile_, uint32_t& k_) -> uint64_t {
