@@ -1,4 +1,5 @@
 """In-tree build of the CUDA library for sm_100a (nvcc cross-compiles without a GPU)."""
+import fcntl
 import os
 import shutil
 import subprocess
@@ -35,8 +36,15 @@ def build(force=False, verbose=False):
     if nvcc is None:
         raise RuntimeError("libequarx.so is missing or out of date and nvcc was not found; "
                            "the CUDA library cannot be built and there is no fallback")
-    tmp = f"{LIB}.{os.getpid()}.tmp"
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + SOURCES
-    subprocess.run(cmd, check=True)
-    os.replace(tmp, LIB)
+    # several processes (one per GPU under torchrun) may import at once: one builds, the others wait
+    with open(LIB + ".lock", "w") as lock:
+        fcntl.flock(lock, fcntl.LOCK_EX)
+        try:
+            if force or is_stale():
+                tmp = f"{LIB}.{os.getpid()}.tmp"
+                cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + SOURCES
+                subprocess.run(cmd, check=True)
+                os.replace(tmp, LIB)
+        finally:
+            fcntl.flock(lock, fcntl.LOCK_UN)
     return LIB
