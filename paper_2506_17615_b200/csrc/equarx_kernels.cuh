@@ -683,14 +683,15 @@ struct FlavourArgs {
     float neg_zero;
 };
 
-// One hop of a chain.  Sender side: the message of v (quantized record or bf16).  Receiver side
-// (the neighbouring lane): v_out = message (+) addend; with a quantized payload one fused multiply-add in fp32,
-// else an fp32 add rounded to bf16 (the BF16 baseline's hop).  `sub` is the lane's position in
-// the tile and flips with every hop.
+// One hop of a chain, in two halves.  chain_send: the message of v (a quantized record, or bf16
+// for an unquantized stage) goes to the FIFO entry (and to the trace), the warp synchronises and
+// the lane moves to the neighbouring position (`sub` flips).  chain_receive: the lane, now acting
+// for the receiving rank, loads the message and folds it into v_io, which holds the addend: with a
+// quantized payload one fused multiply-add in fp32, else an fp32 add rounded to bf16 (the BF16
+// baseline's hop).
 template <int LPB, int PAYLOAD>
-__device__ __forceinline__ void chain_hop(const float (&v)[16], const float (&addend)[16], float (&v_out)[16],
-                                          char* entry, char* trace_rec, uint32_t lane, uint32_t& sub, bool active,
-                                          float neg_zero) {
+__device__ __forceinline__ void chain_send(const float (&v)[16], char* entry, char* trace_rec, uint32_t lane,
+                                           uint32_t& sub, bool active, float neg_zero) {
     if (PAYLOAD != 0) {
         uint4 codes;
         float scale;
@@ -704,24 +705,27 @@ __device__ __forceinline__ void chain_hop(const float (&v)[16], const float (&ad
             if (lane < 8) st_plain_f32(reinterpret_cast<float*>(trace_rec) + lane, hdr);
             if (active) st_plain_128(trace_rec + kRecordHeader + sub * 16, codes);
         }
-        __syncwarp();
-        sub ^= 1u;
+    } else {
+        Vec8 m;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) m.w[i] = pack_bf16x2_rn(v[2 * i], v[2 * i + 1]);
+        if (active) st_fifo_256(entry + sub * 32, m);
+    }
+    __syncwarp();
+    sub ^= 1u;
+}
+
+template <int LPB, int PAYLOAD>
+__device__ __forceinline__ void chain_receive(float (&v_io)[16], const char* entry, uint32_t sub, bool active) {
+    if (PAYLOAD != 0) {
         uint4 c = make_uint4(0, 0, 0, 0);
         float s = 0.0f;
         if (active) {
             c = ld_coherent_128(entry + kRecordHeader + sub * 16);
             s = ld_coherent_f32(reinterpret_cast<const float*>(entry) + sub / LPB);
         }
-#pragma unroll
-        for (int i = 0; i < 16; ++i) v_out[i] = addend[i];
-        dequant_add_payload<PAYLOAD == 0 ? 1 : PAYLOAD>(c, s, v_out);
+        dequant_add_payload<PAYLOAD == 0 ? 1 : PAYLOAD>(c, s, v_io);
     } else {
-        Vec8 m;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) m.w[i] = pack_bf16x2_rn(v[2 * i], v[2 * i + 1]);
-        if (active) st_fifo_256(entry + sub * 32, m);
-        __syncwarp();
-        sub ^= 1u;
         Vec8 r = {};
         if (active) r = ld_fifo_256(entry + sub * 32);
         float y[16];
@@ -729,8 +733,8 @@ __device__ __forceinline__ void chain_hop(const float (&v)[16], const float (&ad
         Vec8 o;
 #pragma unroll
         for (int i = 0; i < 8; ++i)
-            o.w[i] = pack_bf16x2_rn(__fadd_rn(y[2 * i], addend[2 * i]), __fadd_rn(y[2 * i + 1], addend[2 * i + 1]));
-        widen_bf16x16(o, v_out);
+            o.w[i] = pack_bf16x2_rn(__fadd_rn(y[2 * i], v_io[2 * i]), __fadd_rn(y[2 * i + 1], v_io[2 * i + 1]));
+        widen_bf16x16(o, v_io);
     }
 }
 
@@ -754,86 +758,86 @@ __global__ void __launch_bounds__(kPipeThreads) flavour_kernel(const __grid_cons
         char* const trace0 = a.trace ? a.trace + ((uint64_t)k * N * a.tiles_per_shard + t) * kRecordBytes : nullptr;
         uint32_t hops = 0;                                                       // FIFO entry = hops & 1
 
-        auto load_shard = [&](uint32_t rank, uint32_t pos, float (&dst)[16]) {
+        auto fetch = [&](uint32_t rank, uint32_t pos) {                          // a rank's bf16 group at a position
             Vec8 x = {};
             if (active) x = ld_coherent_256(static_cast<const char*>(a.in[rank % N]) + (tile_off + pos * 16) * 2);
-            widen_bf16x16(x, dst);
+            return x;
         };
         auto trace_of = [&](uint32_t event) -> char* {
             return trace0 ? trace0 + (uint64_t)event * a.tiles_per_shard * kRecordBytes : nullptr;
+        };
+        // one hop: v is sent; the receiver's addend is either the prefetched shard xw (then the result
+        // replaces v) or the owner's accumulator acc (then the result replaces acc)
+        auto hop_into_v = [&](float (&v)[16], const Vec8& xw, uint32_t& sub, uint32_t event) {
+            char* entry = fifo + (hops++ & 1u) * kFifoEntryBytes;
+            chain_send<LPB, RS>(v, entry, QRS ? trace_of(event) : nullptr, lane, sub, active, a.neg_zero);
+            widen_bf16x16(xw, v);
+            chain_receive<LPB, RS>(v, entry, sub, active);
+        };
+        auto hop_into_acc = [&](const float (&v)[16], float (&acc)[16], uint32_t& sub, uint32_t event) {
+            char* entry = fifo + (hops++ & 1u) * kFifoEntryBytes;
+            chain_send<LPB, RS>(v, entry, QRS ? trace_of(event) : nullptr, lane, sub, active, a.neg_zero);
+            chain_receive<LPB, RS>(acc, entry, sub, active);
         };
 
         float acc[16];                     // the owner's reduced tile
         uint32_t sub;                      // this lane's position in the tile
         if (!SEMI) {
             sub = lane;
-            load_shard(k + 1, sub, acc);
+            {
+                const Vec8 x0 = fetch(k + 1, sub);
+                widen_bf16x16(x0, acc);
+            }
             for (uint32_t j = 1; j < N; ++j) {                                   // hop into rank k+1+j
-                float x[16];
-                load_shard(k + 1 + j, sub ^ 1u, x);
-                chain_hop<LPB, RS>(acc, x, acc, fifo + (hops & 1u) * kFifoEntryBytes, QRS ? trace_of(j - 1) : nullptr,
-                                    lane, sub, active, a.neg_zero);
-                ++hops;
+                const Vec8 xw = fetch(k + 1 + j, sub ^ 1u);
+                hop_into_v(acc, xw, sub, j - 1);
             }
         } else {
             // chain B: k+h+1 -> ... -> k+N-1 -> owner (h-1 hops); starts at position `lane`
             sub = lane;
-            const uint32_t acc_pos = lane ^ ((h - 1) & 1u);                      // position after B's hops
-            load_shard(k, h >= 2 ? acc_pos : lane, acc);
+            const uint32_t acc_pos = h >= 2 ? lane ^ ((h - 1) & 1u) : lane;      // position after B's hops
+            {
+                const Vec8 xo = fetch(k, acc_pos);
+                widen_bf16x16(xo, acc);
+            }
+            float v[16];
             if (h >= 2) {
-                float v[16];
-                load_shard(k + h + 1, sub, v);
+                {
+                    const Vec8 x0 = fetch(k + h + 1, sub);
+                    widen_bf16x16(x0, v);
+                }
                 for (uint32_t j = 1; j < h; ++j) {
-                    char* entry = fifo + (hops & 1u) * kFifoEntryBytes;
-                    char* tr = QRS ? trace_of(h + j - 1) : nullptr;
                     if (j + 1 < h) {
-                        float x[16];
-                        load_shard(k + h + 1 + j, sub ^ 1u, x);
-                        chain_hop<LPB, RS>(v, x, v, entry, tr, lane, sub, active, a.neg_zero);
+                        const Vec8 xw = fetch(k + h + 1 + j, sub ^ 1u);
+                        hop_into_v(v, xw, sub, h + j - 1);
                     } else {
-                        chain_hop<LPB, RS>(v, acc, acc, entry, tr, lane, sub, active, a.neg_zero);
+                        hop_into_acc(v, acc, sub, h + j - 1);
                     }
-                    ++hops;
                 }
             }
             // chain A: k+h -> k+h-1 -> ... -> k+1 -> owner (h hops); starts so that it ends on acc's position
-            sub = (h >= 2 ? acc_pos : lane) ^ (h & 1u);
-            float v[16];
-            load_shard(k + h, sub, v);
+            sub = acc_pos ^ (h & 1u);
+            {
+                const Vec8 x0 = fetch(k + h, sub);
+                widen_bf16x16(x0, v);
+            }
             for (uint32_t j = 1; j <= h; ++j) {
-                char* entry = fifo + (hops & 1u) * kFifoEntryBytes;
-                char* tr = QRS ? trace_of(j - 1) : nullptr;
                 if (j < h) {
-                    float x[16];
-                    load_shard(k + h - j, sub ^ 1u, x);
-                    chain_hop<LPB, RS>(v, x, v, entry, tr, lane, sub, active, a.neg_zero);
+                    const Vec8 xw = fetch(k + h - j, sub ^ 1u);
+                    hop_into_v(v, xw, sub, j - 1);
                 } else {
-                    chain_hop<LPB, RS>(v, acc, acc, entry, tr, lane, sub, active, a.neg_zero);
+                    hop_into_acc(v, acc, sub, j - 1);
                 }
-                ++hops;
             }
         }
 
         // all-gather: one more message, quantized or bf16, dequantized/forwarded to every rank
-        Vec8 o;
+        Vec8 o = {};
         {
-            char* entry = fifo + (hops & 1u) * kFifoEntryBytes;
+            constexpr int AG = QAG ? PAYLOAD : 0;
+            char* entry = fifo + (hops++ & 1u) * kFifoEntryBytes;
+            chain_send<LPB, AG>(acc, entry, QAG ? trace_of(N - 1) : nullptr, lane, sub, active, a.neg_zero);
             if (QAG) {
-                uint4 codes;
-                float scale;
-                quantize_lane_payload<LPB, PAYLOAD>(acc, codes, scale, a.neg_zero);
-                const uint32_t d = (sub ^ lane) & 1u;
-                float hdr = __shfl_sync(0xFFFFFFFFu, scale, ((lane * LPB) & 31u) ^ d);
-                if (lane >= 32u / LPB) hdr = 0.0f;
-                char* tr = trace_of(N - 1);
-                if (lane < 8) st_plain_f32(reinterpret_cast<float*>(entry) + lane, hdr);
-                if (active) st_plain_128(entry + kRecordHeader + sub * 16, codes);
-                if (tr) {
-                    if (lane < 8) st_plain_f32(reinterpret_cast<float*>(tr) + lane, hdr);
-                    if (active) st_plain_128(tr + kRecordHeader + sub * 16, codes);
-                }
-                __syncwarp();
-                sub ^= 1u;
                 uint4 c = make_uint4(0, 0, 0, 0);
                 float s = 0.0f;
                 if (active) {
@@ -841,17 +845,9 @@ __global__ void __launch_bounds__(kPipeThreads) flavour_kernel(const __grid_cons
                     s = ld_coherent_f32(reinterpret_cast<const float*>(entry) + sub / LPB);
                 }
                 o = dequant_to_bf16_payload<PAYLOAD>(c, s);
-            } else {
-                Vec8 m;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) m.w[i] = pack_bf16x2_rn(acc[2 * i], acc[2 * i + 1]);
-                if (active) st_fifo_256(entry + sub * 32, m);
-                __syncwarp();
-                sub ^= 1u;
-                o = Vec8{};
-                if (active) o = ld_fifo_256(entry + sub * 32);
+            } else if (active) {
+                o = ld_fifo_256(entry + sub * 32);
             }
-            ++hops;
         }
         if (active) {
             const uint64_t byte_off = (tile_off + sub * 16) * 2;
