@@ -345,3 +345,47 @@ def test_every_sweep_point_sampled(gu, nranks, block, dist):
         assert torch.equal(out.view(torch.int16), out2.view(torch.int16)), w.name
         del out, out2, x
         torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_offsets_beyond_four_gigabytes(gu, variant):
+    """Two ranks of 2^31 + 1024 elements each (4.3 GB per tensor): element and byte offsets pass 2^32.
+    Sampled blocks, including the last blocks of both shards, against the oracle."""
+    n, block = 2, 512
+    count = (1 << 31) + 2 * 512
+    g = torch.Generator(device="cuda").manual_seed(99)
+    x = torch.empty((n, count), dtype=torch.bfloat16, device="cuda")
+    for r in range(n):
+        x[r].normal_(generator=g)
+    out, _ = gu.run_sim(x, block, variant=variant)
+    bps = count // n // block
+    picks = gu.sample_blocks(n, bps, 16, seed=3)
+    exp = gu.oracle_out_on_samples(x, picks, block)
+    gu.assert_same_words(gu.gather_blocks(out, picks, block), exp, variant)
+    assert torch.equal(out[0].view(torch.int16), out[1].view(torch.int16))
+    del out, x
+    torch.cuda.empty_cache()
+
+
+def test_runs_on_the_stream_it_is_given(gu):
+    """The work is enqueued on the caller's stream: issued on a side stream behind a long-running
+    fill of the input, it must see the filled input, and the default stream must stay idle."""
+    n, block = 4, 256
+    count = n * block * 64
+    side = torch.cuda.Stream()
+    x = torch.zeros((n, count), dtype=torch.bfloat16, device="cuda")
+    src = wl.make_inputs(wl.Workload("t", n, count, block, "normal", seed=31)).cuda()
+    out = torch.empty_like(x)
+    wb = eq.allreduce_sim_pipelined_workspace_bytes(n, count, block, False)
+    ws = torch.empty(wb, dtype=torch.uint8, device="cuda")
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        big = torch.empty(1 << 28, dtype=torch.float32, device="cuda")
+        for _ in range(8):
+            big.fill_(1.0)                 # keeps the side stream busy for a while
+        x.copy_(src)                       # the inputs only become valid behind that work
+        eq.allreduce_sim_pipelined([x[r] for r in range(n)], [out[r] for r in range(n)], n, count, block, ws, wb,
+                                   False, side.cuda_stream)
+    side.synchronize()
+    exp = oracle.allreduce(wl.as_u16(src), block)["out"]
+    gu.assert_same_words(out, exp, "side stream")
