@@ -5,8 +5,6 @@ import ctypes
 import os
 import re
 
-import pytest
-
 import paper_2506_17615_b200 as eq
 from paper_2506_17615_b200 import binding
 
