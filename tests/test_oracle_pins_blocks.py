@@ -70,7 +70,7 @@ def test_hand_chain_intermediate_sum():
     assert np.array_equal(c1, expect)
 
 
-@pytest.mark.parametrize("case", ["ties", "spike"])
+@pytest.mark.parametrize("case", ["ties", "spike", "reciprocal_of_amax"])
 def test_hand_value_blocks(case):
     g = GOLD[case]
     x = bf16_words(g["x"])
