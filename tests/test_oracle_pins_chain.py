@@ -215,3 +215,23 @@ def test_paper_mse_full_loop():
     bf16_noise = _mse_vs(base[0], res["exact_sum"])
     assert abs(mse_exact - (pred + np.mean(res["exact_sum"] ** 2) * 2.0 ** -18 / 3)) < 0.1 * mse_exact, (mse_exact, pred)
     assert bf16_noise < 0.15 * mse_exact
+
+
+def test_step_functions_compose_to_the_ring():
+    """quantize_blocks -> rs_step x (N-1) -> ag_dequant along every shard's chain reproduces the
+    ring simulation's trace and outputs: the stand-alone step functions carry the same arithmetic
+    (in particular the single-rounding multiply-add of the hop, which the rational brute force pins
+    on the ring)."""
+    N, B = 5, 64
+    w = wl.Workload("t", N, N * B * 7, B, "normal", seed=13)
+    x = wl.as_u16(wl.make_inputs(w))
+    res = oracle.allreduce(x, B, trace=True)
+    shard = x.shape[1] // N
+    for k in range(N):
+        sl = slice(k * shard, (k + 1) * shard)
+        codes, scales = oracle.quantize_blocks(x[(k + 1) % N, sl], B)
+        for j in range(N):
+            assert np.array_equal(codes, res["codes"][k, j]) and np.array_equal(scales, res["scales"][k, j]), (k, j)
+            if j + 1 < N:
+                codes, scales = oracle.rs_step(codes, scales, x[(k + 2 + j) % N, sl], B)
+        assert np.array_equal(oracle.ag_dequant(codes, scales, B), res["out"][0, sl])
