@@ -9,6 +9,10 @@
  *   - extern "C"; returns an EQUARX_* status; never throws, aborts or exits.
  *   - Arguments are validated on the host first; on a validation error
  *     nothing is launched and no CUDA call is made.
+ *   - A failing launch is reported as EQUARX_ERR_CUDA (the CUDA error code is kept for
+ *     equarx_last_cuda_error()); the launches that preceded it in the same call stay
+ *     enqueued.  For tests, EQUARX_INJECT_LAUNCH_ERROR=<code> in the environment makes
+ *     every launch report that code without launching anything.
  *   - Work is enqueued on `stream` and the call returns without
  *     synchronising.  Device buffers must stay valid until the stream has
  *     reached the work.  The library allocates and frees nothing: the caller

@@ -58,6 +58,14 @@ bool use_pdl() {
     return on;
 }
 
+// Host-side fault injection for tests: with EQUARX_INJECT_LAUNCH_ERROR=<cudaError_t value> in the
+// environment every launch is skipped and reports that error instead, so that the error path
+// (status, equarx_last_cuda_error) can be exercised without making a GPU fault.
+inline cudaError_t injected_launch_error() {
+    const char* e = std::getenv("EQUARX_INJECT_LAUNCH_ERROR");
+    return e ? cudaError_t(std::atoi(e)) : cudaSuccess;
+}
+
 template <typename Kernel, typename Args>
 int launch(Kernel kernel, dim3 grid, const Args& args, cudaStream_t stream, bool dependent) {
     cudaLaunchConfig_t cfg = {};
@@ -70,7 +78,8 @@ int launch(Kernel kernel, dim3 grid, const Args& args, cudaStream_t stream, bool
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = (dependent && use_pdl()) ? 1 : 0;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, args);
+    cudaError_t e = injected_launch_error();
+    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, kernel, args);
     if (e != cudaSuccess) {
         g_last_cuda_error = int(e);
         (void)cudaGetLastError();
@@ -395,7 +404,8 @@ int equarx_allreduce_sim_pipelined(const void* const* in_bf16, void* const* out_
     cfg.attrs = attr;
     cfg.numAttrs = use_pdl() ? 1 : 0;
     void* params[1] = {&a};
-    e = cudaLaunchKernelExC(&cfg, kernel, params);
+    e = injected_launch_error();
+    if (e == cudaSuccess) e = cudaLaunchKernelExC(&cfg, kernel, params);
     if (e != cudaSuccess) {
         g_last_cuda_error = int(e);
         (void)cudaGetLastError();
@@ -476,7 +486,8 @@ int equarx_allreduce_sim_flavour(const void* const* in_bf16, void* const* out_bf
         }
     }
     void* params[1] = {&a};
-    e = cudaLaunchKernel(kernel, dim3(unsigned(ctas)), dim3(kPipeThreads), params, 0, stream);
+    e = injected_launch_error();
+    if (e == cudaSuccess) e = cudaLaunchKernel(kernel, dim3(unsigned(ctas)), dim3(kPipeThreads), params, 0, stream);
     if (e != cudaSuccess) {
         g_last_cuda_error = int(e);
         (void)cudaGetLastError();

@@ -8,7 +8,7 @@ import torch
 
 import oracle
 import paper_2506_17615_b200 as eq
-from paper_2506_17615_b200 import workloads as wl
+from paper_2506_17615_b200 import binding, workloads as wl
 
 pytestmark = pytest.mark.gpu
 
@@ -389,3 +389,34 @@ def test_runs_on_the_stream_it_is_given(gu):
     side.synchronize()
     exp = oracle.allreduce(wl.as_u16(src), block)["out"]
     gu.assert_same_words(out, exp, "side stream")
+
+
+def test_launch_errors_are_reported_not_raised_on_the_gpu(gu, monkeypatch):
+    """A failing launch (injected on the host: no kernel runs, the GPU is not touched) comes back
+    as EQUARX_ERR_CUDA with the CUDA error code available, from every kind of entry point, and
+    the library works again afterwards."""
+    n, block = 4, 256
+    count = n * block * 4
+    x = wl.make_inputs(wl.Workload("t", n, count, block, "normal", seed=1)).cuda()
+    out = torch.empty_like(x)
+    ins, outs = [x[r] for r in range(n)], [out[r] for r in range(n)]
+    wb = max(eq.allreduce_sim_workspace_bytes(n, count, block), eq.allreduce_sim_pipelined_workspace_bytes(n, count, block),
+             eq.allreduce_sim_flavour_workspace_bytes(n, count, block, 7))
+    ws = torch.empty(wb, dtype=torch.uint8, device="cuda")
+    codes = torch.empty(count, dtype=torch.int8, device="cuda")
+    scales = torch.empty(count // block, device="cuda")
+    s = gu.stream_handle()
+    monkeypatch.setenv("EQUARX_INJECT_LAUNCH_ERROR", "719")          # cudaErrorLaunchFailure
+    calls = [lambda: eq.allreduce_sim(ins, outs, n, count, block, ws, wb, False, s),
+             lambda: eq.allreduce_sim_pipelined(ins, outs, n, count, block, ws, wb, False, s),
+             lambda: eq.allreduce_sim_flavour(ins, outs, n, count, block, 7, ws, wb, False, s),
+             lambda: eq.quantize_blocks(x[0], count, block, codes, scales, s),
+             lambda: eq.allreduce_sim_static(ins, outs, n, count, block, s)]
+    for call in calls:
+        with pytest.raises(eq.EquarxError) as err:
+            call()
+        assert err.value.status == binding.ERR_CUDA and eq.last_cuda_error() == 719
+    monkeypatch.delenv("EQUARX_INJECT_LAUNCH_ERROR")
+    eq.allreduce_sim_pipelined(ins, outs, n, count, block, ws, wb, False, s)
+    torch.cuda.synchronize()
+    gu.assert_same_words(out, oracle.allreduce(wl.as_u16(x.cpu()), block)["out"], "after the injected failures")
