@@ -160,9 +160,10 @@ def run_reference(args):
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "int8 codes, fp32 accumulate, bf16 in/out",
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic", "config": {"workload": w.name, "nranks": w.nranks, "count_per_rank": count,
-                                        "block": w.block, "dist": w.dist},
+                                        "block": w.block, "dist": w.dist, "payload": "int8 codes + fp32 block scales",
+                                        "io": "bf16"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -446,9 +447,9 @@ def main():
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "int8 codes, fp32 accumulate, bf16 in/out", "data": "synthetic",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "nranks": N, "count_per_rank": count, "block": block, "dist": w.dist,
-                       "bytes_per_rank": 2 * count, "parallelism": f"replicas x{world}" if world > 1 else "1 GPU",
+                       "bytes_per_rank": 2 * count, "payload": "int8 codes + fp32 block scales", "io": "bf16", "parallelism": f"replicas x{world}" if world > 1 else "1 GPU",
                        "l2": f"{sets} input/output sets used in rotation ({sets * 2 * in_bytes / 1e6:.0f} MB "
                              f"working set against a 126 MB L2); no explicit flush",
                        "pdl_between_step_launches": os.environ.get("EQUARX_PDL", "1") != "0"},
