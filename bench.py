@@ -55,6 +55,12 @@ def workload_by_name(name):
     return table[name]
 
 
+def base_config(w):
+    """The workload description shared by both arms of the bench."""
+    return {"workload": w.name, "nranks": w.nranks, "count_per_rank": w.count, "block": w.block, "dist": w.dist,
+            "bytes_per_rank": 2 * w.count, "payload": "int8 codes + fp32 block scales", "io": "bf16"}
+
+
 def algorithmic_bytes(n_ranks, count, block):
     """Minimum bytes the schedule moves: N bf16 reads, every hop message written and read
     once (N messages of count*(1+4/block) bytes each way), N bf16 writes."""
@@ -161,9 +167,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-        "data": "synthetic", "config": {"workload": w.name, "nranks": w.nranks, "count_per_rank": count,
-                                        "block": w.block, "dist": w.dist, "payload": "int8 codes + fp32 block scales",
-                                        "io": "bf16"},
+        "data": "synthetic", "config": dict(base_config(w), sample_count_per_rank=count),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -448,8 +452,7 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": w.name, "nranks": N, "count_per_rank": count, "block": block, "dist": w.dist,
-                       "bytes_per_rank": 2 * count, "payload": "int8 codes + fp32 block scales", "io": "bf16", "parallelism": f"replicas x{world}" if world > 1 else "1 GPU",
+            "config": {**base_config(w), "parallelism": f"replicas x{world}" if world > 1 else "1 GPU",
                        "l2": f"{sets} input/output sets used in rotation ({sets * 2 * in_bytes / 1e6:.0f} MB "
                              f"working set against a 126 MB L2); no explicit flush",
                        "pdl_between_step_launches": os.environ.get("EQUARX_PDL", "1") != "0"},
