@@ -82,7 +82,9 @@ __device__ __forceinline__ void st_scale(float* p, float v, uint64_t pol) {
 }
 
 // Accessors for data that is written and read inside the SAME launch (the pipelined
-// kernel): no read-only (.nc) path, L2 only.
+// kernels): no read-only (.nc) path.  A record is always stored by the lanes of a warp and,
+// after a __syncwarp, loaded by lanes of the same warp, so the loads may use the default
+// (L1-allocating) path: the SM's own stores keep its L1 consistent.
 __device__ __forceinline__ Vec8 ld_coherent_256(const void* p) {
     Vec8 r;
     asm volatile(
@@ -113,7 +115,7 @@ __device__ __forceinline__ void st_fifo_256(void* p, const Vec8& r) {
 
 __device__ __forceinline__ uint4 ld_coherent_128(const void* p) {
     uint4 r;
-    asm volatile("ld.global.cg.v4.b32 {%0,%1,%2,%3}, [%4];"
+    asm volatile("ld.global.ca.v4.b32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
                  : "l"(p)
                  : "memory");
@@ -122,7 +124,7 @@ __device__ __forceinline__ uint4 ld_coherent_128(const void* p) {
 
 __device__ __forceinline__ float ld_coherent_f32(const float* p) {
     float r;
-    asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(r) : "l"(p) : "memory");
+    asm volatile("ld.global.ca.f32 %0, [%1];" : "=f"(r) : "l"(p) : "memory");
     return r;
 }
 
