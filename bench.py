@@ -330,8 +330,8 @@ def main():
                 "algorithmic_bytes_per_launch": alg_bytes,
                 "dram_gbs": traffic / (ms_step * 1e-3) / 1e9, "dram_frac": traffic / (ms_step * 1e-3) / 1e9 / peak,
                 "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "note": "hop messages are produced and consumed in L2, so DRAM traffic (inputs + outputs) is "
-                        "below the algorithmic bytes and frac can exceed 1"}
+                "note": "hop messages are written through to L2 and consumed at once from the SM's L1/L2, so DRAM "
+                        "traffic (inputs + outputs) is below the algorithmic bytes and frac can exceed 1"}
 
     # ---- the same work as one launch per ring step
     ms_steps = timed(step_by_steps, args.steps)

@@ -169,7 +169,7 @@ int equarx_allreduce_sim_range(const void *const *in_bf16, void *const *out_bf16
  * waiting for the rest of the shard.  Every hop message is still written to
  * memory as a record and read back from there (by the neighbouring lane, acting
  * for the receiving rank), but it is consumed right after it was produced and is
- * therefore served from L2 instead of HBM.  Outputs, and with keep_trace the
+ * therefore served from the SM's L1/L2 instead of HBM.  Outputs, and with keep_trace the
  * whole trace, are identical to equarx_allreduce_sim bit for bit; only the order
  * in which tiles advance differs.
  *
