@@ -68,3 +68,19 @@ def test_reference_arm_prints_one_line_and_other_ranks_stay_silent():
     line = json.loads(out.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["unit"] == "GB/s" and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_sweep_summary_from_a_results_file(tmp_path):
+    """The sweep's markdown summary is plain host code: feed it two fabricated result lines."""
+    from paper_2506_17615_b200 import sweep
+    rows = []
+    for nbytes, frac in ((1 << 20, 0.4), (1 << 26, 1.3)):
+        leg = {"ms": 1.0, "gbs_in": 1000.0, "frac": frac}
+        rows.append({"nranks": 8, "bytes_per_rank": nbytes, "block": 256, "dist": "normal", "iters": 5, "sets": 2,
+                     "pipelined": leg, "by_steps": dict(leg, frac=frac * 0.75), "bf16_sim": leg,
+                     "peak_gbs": 6534.1, "peak_source": "measured"})
+    path = tmp_path / "sweep.jsonl"
+    path.write_text("\n".join(json.dumps(r) for r in rows) + "\n")
+    text = sweep.summarize(str(path))
+    assert "| 8 | 256 | 1 MB | 1000 (0.400)" in text and "| 8 | 256 | 64 MB | 1000 (1.300)" in text
+    assert "All 1 points with at least 64 MB per rank: pipelined 1.300 - 1.300" in text
