@@ -121,3 +121,75 @@ def chain_allreduce(words, block, payload="int8"):
             for c, i in zip(codes, idx):
                 out[i] = bf16_word(bf16(f32(c * scale)))
     return out, events
+
+
+def _quantize(v, payload):
+    """(scale, code VALUES as Fractions) for any payload."""
+    if payload == "int8":
+        scale, codes = quantize_block(v)
+        return scale, [Fraction(c) for c in codes]
+    return quantize_block_fp8(v, payload)
+
+
+def tree_allreduce(words, block, semi, quant_rs, quant_ag, payload="int8"):
+    """The adder chain of Fig. 4 (semi = False) or the adder tree of Fig. 5 (semi = True) of
+    every shard, with or without quantized reduce-scatter hops and all-gather (Section 3.4).
+
+    A hop is `send(v)` followed by `receive(message, addend)`:
+      quantized  : message = (scale, codes) of v; result = f32(code * scale + addend), ONE rounding,
+                   and the result stays an fp32 value until it is sent again;
+      unquantized: message = bf16(v); result = bf16(message + addend).
+    Semi loop, shard k, h = N/2 (Section 3.3: on four devices 2 -> 1 -> 0 and 3 -> 0):
+      chain A: k+h -> k+h-1 -> ... -> k+1 -> owner k      (h hops, events 0..h-1)
+      chain B: k+h+1 -> k+h+2 -> ... -> k-1 -> owner k    (h-1 hops, events h..N-2)
+      B is one hop shorter, so its partial reaches the owner first: the owner holds its own shard,
+      receives B's message, then A's.
+    All-gather: one more quantize/dequantize pair (event N-1), or a plain bf16 rounding.
+    Returns (out_words, events) with events[(k, b, j)] = (scale, code values).  Rationals have no
+    signed zero: a result that is -0.0 in IEEE arithmetic comes back as the word 0x0000.
+    """
+    n_ranks = len(words)
+    count = len(words[0])
+    shard = count // n_ranks
+    h = n_ranks // 2
+    out = [0] * count
+    events = {}
+    for k in range(n_ranks):
+        for b in range(shard // block):
+            idx = [k * shard + b * block + i for i in range(block)]
+
+            def x(rank):
+                return [frac_from_bf16_word(words[rank % n_ranks][i]) for i in idx]
+
+            def hop(v, addend, event):
+                if quant_rs:
+                    scale, vals = _quantize(v, payload)
+                    events[(k, b, event)] = (scale, vals)
+                    return [f32(c * scale + a) for c, a in zip(vals, addend)]
+                return [bf16(bf16(t) + a) for t, a in zip(v, addend)]
+
+            if not semi:
+                v = x(k + 1)
+                for j in range(1, n_ranks):
+                    v = hop(v, x(k + 1 + j), j - 1)
+                acc = v
+            else:
+                acc = x(k)                                  # the owner's own shard
+                if h >= 2:                                  # chain B, received first
+                    v = x(k + h + 1)
+                    for j in range(1, h - 1):
+                        v = hop(v, x(k + h + 1 + j), h + j - 1)
+                    acc = hop(v, acc, n_ranks - 2)
+                v = x(k + h)                                # chain A, received second
+                for j in range(1, h):
+                    v = hop(v, x(k + h - j), j - 1)
+                acc = hop(v, acc, h - 1)
+            if quant_ag:
+                scale, vals = _quantize(acc, payload)
+                events[(k, b, n_ranks - 1)] = (scale, vals)
+                res = [bf16(f32(c * scale)) for c in vals]
+            else:
+                res = [bf16(t) for t in acc]
+            for r, i in zip(res, idx):
+                out[i] = bf16_word(r)
+    return out, events

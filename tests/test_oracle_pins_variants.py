@@ -218,3 +218,34 @@ def test_fp8_error_is_larger_than_int8_and_ordered():
         d = to_f64(oracle.allreduce_variant(x, 64, False, True, True, payload=fmt)["out"][0]) - exact
         mse[fmt] = float(np.mean(d * d))
     assert mse["int8"] < mse["e4m3"] < mse["e5m2"]
+
+
+# ---------------------------------------------------------------- adder tree, bit for bit
+def _fp8_or_int(c, payload):
+    return float(int(c)) if payload == "int8" else _fp8_value(int(c) & 0xFF, payload)
+
+
+@pytest.mark.parametrize("payload", ["int8", "e4m3", "e5m2"])
+@pytest.mark.parametrize("kind", ["normal", "wide", "halves", "tiny"])
+@pytest.mark.parametrize("semi,qr,qa", FLAVOURS)
+@pytest.mark.parametrize("nranks,block,bps", [(2, 4, 1), (4, 3, 2), (6, 5, 1), (8, 2, 1)])
+def test_adder_tree_exact_rational(payload, kind, semi, qr, qa, nranks, block, bps):
+    """Fig. 4 / Fig. 5 evaluated with rationals and one explicit rounding per IEEE operation
+    (tests/exact_fp.py, written from the figures) must give the oracle's scales, codes and outputs
+    bit for bit: in particular the semi-loop owner, which adds chain B's message to its own shard,
+    then chain A's, each by one fused multiply-add, and stays in fp32 in between."""
+    if payload != "int8" and not (qr or qa):
+        pytest.skip("nothing is quantized: the payload does not matter")
+    from test_oracle_pins_chain import rand_bf16
+    from exact_fp import f32_word, tree_allreduce
+    rng = np.random.default_rng(hash((payload, kind, semi, qr, qa, nranks, block)) % (2 ** 32))
+    x = rand_bf16(rng, (nranks, nranks * block * bps), kind)
+    res = oracle.allreduce_variant(x, block, semi, qr, qa, trace=True, payload=payload)
+    out, events = tree_allreduce([[int(w) for w in row] for row in x], block, semi, qr, qa, payload)
+    for r in range(nranks):
+        assert [0 if int(w) == 0x8000 else int(w) for w in res["out"][r]] == out
+    assert len(events) == ((nranks - 1 if qr else 0) + (1 if qa else 0)) * nranks * bps
+    for (k, b, j), (scale, vals) in events.items():
+        assert int(res["scales"][k, j, b].view(np.uint32)) == f32_word(scale), (k, b, j)
+        got = [_fp8_or_int(c, payload) for c in res["codes"][k, j, b * block:(b + 1) * block]]
+        assert got == [float(v) for v in vals], (k, b, j)
