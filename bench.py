@@ -3,16 +3,23 @@
 
 One "step" is one pass of the whole hot path -- ring step 0 (quantize), N-1
 dequantize-add-requantize steps and the all-gather dequantize -- over one
-batch of synthetic bf16 tensors, through the C ABI (equarx_allreduce_sim).
+batch of synthetic bf16 tensors, through the C ABI.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C2] [--impl ours|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C3] [--impl ours|reference]
 
 Prints ONE JSON line.  `value` is GB/s of bf16 input reduced (2 * count *
-nranks bytes per step) with inputs resident in device memory; `e2e` is the
-same metric with pinned host buffers and the copies inside the timed region.
-With --gpus N > 1 (under torchrun) every rank runs an independent replica
-on its own GPU (the path has no inter-GPU exchange): weak scaling, no
-collective on the data path; NCCL is used for the barrier and the max only.
+nranks bytes per step) with inputs resident in device memory, for the
+single-launch (chain-fused) schedule; `by_steps` is the same work as one launch
+per ring step, whose hop messages do travel through memory.  Each schedule
+carries its own roofline: bytes it must move / CUDA-event time / measured HBM
+peak.  `e2e` is the same metric through equarx_allreduce_sim_host: pinned host
+buffers, the copies inside the timed region.  A train of K steps is timed
+between CUDA events; trains are repeated until at least MIN_TIMED_SECONDS of
+GPU time has been measured and the median train is reported.
+
+With --gpus N > 1 (under torchrun) every rank runs an independent replica on
+its own GPU (the path has no inter-GPU exchange): weak scaling, no collective
+on the data path; NCCL carries the barrier and the max only.
 `--impl reference` times the CPU oracle on a bounded sample instead.
 """
 import argparse
@@ -32,15 +39,22 @@ METRIC = "q-AllReduce GB/s (bf16 in) & % of HBM roofline on 1 B200, N simulated 
 UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+MIN_TIMED_SECONDS = 0.5
+L2_BYTES = 126_000_000
 
-# DRAM traffic of one dequantize-add-requantize launch per element of a rank's shard,
-# from the ncu capture summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum
-# divided by the elements per rank; cold L2, so both inputs come from DRAM and the outgoing
-# message stays in L2).
-DAR_TRAFFIC_BYTES_PER_ELEMENT = 3.017
-# DRAM traffic of one pipelined launch per element of every rank (ncu, profiles/): the N inputs
-# are read once and the N outputs written once; hop messages never leave L2.
-PIPELINED_TRAFFIC_BYTES_PER_RANK_ELEMENT = 4.0
+# DRAM traffic measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum per launch, divided
+# by the elements the launch processes: count*nranks for the whole AllReduce, count for one ring
+# step), from the captures summarised under profiles/.  Traffic grows in proportion to the elements
+# processed, so a full launch of another size is this figure times its elements.  Hop launches: the
+# outgoing message stays in L2 while a step's messages (count * (1 + 4/block) bytes over all ranks)
+# fit the part of L2 that keeps them, about 20 MB; above that it is written back and read again
+# from DRAM.
+NCU_TRAFFIC = {
+    "chain_fused_kernel": {"bytes_per_element": 4.0, "profile": "profiles/chain_fused_kernel_c2_c3.md"},
+    "rs_step_hop_small": {"bytes_per_element": 3.017, "profile": "profiles/rs_step_kernel_c2_full.md"},
+    "rs_step_hop_large": {"bytes_per_element": 3.95, "profile": "profiles/rs_step_kernel_c2_full.md"},
+}
+HOP_MESSAGES_STAY_IN_L2_BYTES = 20_000_000
 
 
 def workload_by_name(name):
@@ -55,17 +69,35 @@ def workload_by_name(name):
     return table[name]
 
 
-def base_config(w):
-    """The workload description shared by both arms of the bench."""
+def input_sets(w):
+    """How many input/output sets the timed steps rotate through, so that no step finds its
+    inputs in L2: one set if a step's inputs alone exceed L2 several times over."""
+    in_bytes = 2 * w.count * w.nranks
+    return 1 if in_bytes > 1_000_000_000 else min(64, max(2, -(-3 * L2_BYTES // (2 * in_bytes))))
+
+
+def base_config(w, world):
+    """The workload description; identical for both arms of the bench."""
+    sets = input_sets(w)
+    in_bytes = 2 * w.count * w.nranks
     return {"workload": w.name, "nranks": w.nranks, "count_per_rank": w.count, "block": w.block, "dist": w.dist,
-            "bytes_per_rank": 2 * w.count, "payload": "int8 codes + fp32 block scales", "io": "bf16"}
+            "bytes_per_rank": 2 * w.count, "payload": "int8 codes + fp32 block scales", "io": "bf16",
+            "parallelism": f"replicas x{world}" if world > 1 else "1 GPU",
+            "l2": f"{sets} input/output set(s) used in rotation ({sets * 2 * in_bytes / 1e6:.0f} MB working set "
+                  f"against a 126 MB L2); no explicit flush"}
 
 
-def algorithmic_bytes(n_ranks, count, block):
-    """Minimum bytes the schedule moves: N bf16 reads, every hop message written and read
-    once (N messages of count*(1+4/block) bytes each way), N bf16 writes."""
+def ring_schedule_bytes(n_ranks, count, block):
+    """Minimum bytes the ring schedule moves: N bf16 reads, every hop message written and read
+    once (N messages of count*(1+4/block) bytes each way), N bf16 writes: n*N*(6 + 8/B)."""
     wire = count * (1.0 + 4.0 / block)
     return 2.0 * count * n_ranks + 2.0 * n_ranks * wire + 2.0 * count * n_ranks
+
+
+def chain_fused_bytes(n_ranks, count):
+    """Bytes the single-launch chain-fused form must move: every input read once, every output
+    written once (its hop messages never leave the registers): 4*n*N."""
+    return 4.0 * count * n_ranks
 
 
 def launch_bytes(kind, n_ranks, count, block):
@@ -83,7 +115,7 @@ def hbm_peak():
         with open(path) as f:
             return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
     except Exception:
-        return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
+        return FALLBACK_HBM_GBS, "fallback (no MEASURED_PEAKS.json: 6650 GB/s, an earlier B200 copy measurement)"
 
 
 class ClockSampler:
@@ -137,6 +169,16 @@ class ClockSampler:
                 "reasons": reasons, "samples": len(rows), "total_samples": len(self.samples)}
 
 
+def _gcd(a, b):
+    while b:
+        a, b = b, a % b
+    return a
+
+
+def _lcm(a, b):
+    return a // _gcd(a, b) * b
+
+
 def run_reference(args):
     """The CPU oracle, as it stands, on the host cores: bounded sample per step."""
     rank = int(os.environ.get("RANK", "0"))
@@ -144,6 +186,7 @@ def run_reference(args):
         return
     import oracle
     from paper_2506_17615_b200 import workloads as wl
+    world = int(os.environ.get("WORLD_SIZE", "1"))
     w = workload_by_name(args.workload)
     unit = _lcm(w.hidden, w.nranks * w.block) if w.hidden else w.nranks * w.block   # whole token rows
     # calibrate on the smallest sample, then size a step so that the run ends in ~2 minutes
@@ -162,52 +205,66 @@ def run_reference(args):
         oracle.allreduce(x, w.block)
     dt = (time.perf_counter() - t0) / args.steps
     value = 2.0 * count * w.nranks / dt / 1e9
-    sample = f"first {count} of {w.count} elements per rank of {w.name} ({count * w.nranks} element-hops per step)"
+    sample = (f"first {count} of {w.count} elements per rank of {w.name} ({count * w.nranks} element-hops per "
+              f"step), single thread")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-        "data": "synthetic", "config": dict(base_config(w), sample_count_per_rank=count),
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "data": "synthetic", "config": base_config(w, world),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+                         "host_cores": os.cpu_count()},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line))
 
 
-def _gcd(a, b):
-    while b:
-        a, b = b, a % b
-    return a
+def cpu_baseline_and_parity(w, x_dev, out_dev):
+    """The oracle on a bounded sample of the bench workload, on the host's cores, and, from the same
+    oracle run, the parity verdict of the GPU outputs `out_dev` for the inputs `x_dev` ([N, count]).
 
-
-def _lcm(a, b):
-    return a // _gcd(a, b) * b
-
-
-def cpu_baseline(w):
-    """The oracle on a bounded sample of the bench workload, on this machine's host cores."""
+    The sample is the whole workload when the oracle finishes it in about half a minute; else a set
+    of whole blocks drawn from every shard (blocks are independent, so they form a smaller AllReduce
+    whose outputs must equal the full problem's outputs at those blocks)."""
+    import numpy as np
+    import torch
     import oracle
     from paper_2506_17615_b200 import workloads as wl
-    count = w.count
-    # ~60 M element-hops per second on one core: keep the sample near 10-30 s
-    max_events = 600_000_000
-    if count * w.nranks > max_events:
-        unit = _lcm(w.hidden, w.nranks * w.block) if w.hidden else w.nranks * w.block
-        count = max(unit, max_events // w.nranks // unit * unit)
-    x = wl.as_u16(wl.make_inputs(w, count=count))
-    oracle.allreduce(x[:, :w.nranks * w.block], w.block)      # loads the library
-    reps, t_total = 0, 0.0
+    n, count, block = w.nranks, w.count, w.block
+    max_events = 600_000_000                       # ~60 M element-hops per second on one core
+    if count * n <= max_events:
+        x = wl.as_u16(x_dev)
+        got = wl.as_u16(out_dev)
+        part = "the full workload"
+    else:
+        shard = count // n
+        bps = shard // block
+        m = max(1, min(bps, max_events // (n * n * block)))
+        g = torch.Generator().manual_seed(12345)
+        idx = []
+        for k in range(n):
+            pick = torch.randperm(bps, generator=g)[:m].sort().values
+            idx.append((k * shard + pick[:, None] * block + torch.arange(block)[None, :]).reshape(-1))
+        idx = torch.cat(idx).to(x_dev.device)
+        x = wl.as_u16(x_dev[:, idx])
+        got = wl.as_u16(out_dev[:, idx])
+        part = f"{m} of {bps} blocks of every shard ({n * m * block} of {count} elements per rank)"
+    oracle.allreduce(x[:, :n * block], block)      # loads the library
+    reps, t_total, res = 0, 0.0, None
     while t_total < 10.0 and reps < 20:
         t0 = time.perf_counter()
-        oracle.allreduce(x, w.block)
+        res = oracle.allreduce(x, block)
         t_total += time.perf_counter() - t0
         reps += 1
     dt = t_total / reps
-    part = "the full workload" if count == w.count else f"the first {count} of {w.count} elements per rank"
-    return {"value": 2.0 * count * w.nranks / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+    bad = int(np.count_nonzero(got != res["out"]))
+    base = {"value": 2.0 * x.shape[1] * n / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
             "sample": f"{part} of {w.name}, {reps} passes, {dt:.3f} s per pass, single thread",
             "host_cores": os.cpu_count()}
+    parity = {"against": "oracle", "checked_words": int(got.size), "of_words": n * count, "mismatches": bad,
+              "verdict": "bit-exact" if bad == 0 else "MISMATCH", "sample": part}
+    return base, parity
 
 
 def max_over_ranks(ms, world, device):
@@ -228,18 +285,29 @@ def aggregate_value(bytes_per_rank_step, ms_step, world):
     return world * bytes_per_rank_step / (ms_step * 1e-3) / 1e9
 
 
+def roofline_entry(kernel, bytes_per_launch, ms_per_launch, peak, peak_src, traffic, traffic_src, model):
+    achieved = bytes_per_launch / (ms_per_launch * 1e-3) / 1e9
+    return {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
+            "frac": achieved / peak, "traffic": traffic, "traffic_source": traffic_src,
+            "bytes_per_launch": bytes_per_launch, "bytes_model": model, "peak_source": peak_src,
+            "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
-    ap.add_argument("--workload", default="C2")
+    ap.add_argument("--workload", default="C3")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the flavours and the bf16 comparator")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
+    if args.steps < 1:
+        args.steps = 1
     if args.impl == "reference":
         run_reference(args)
         return
@@ -279,22 +347,24 @@ def main():
     w = workload_by_name(args.workload)
     N, count, block = w.nranks, w.count, w.block
     in_bytes = 2 * count * N
-    # inputs of consecutive steps differ, so no step finds its inputs in the 126 MB L2
-    sets = 1 if in_bytes > 1_000_000_000 else min(64, max(2, -(-378_000_000 // (2 * in_bytes))))
-    ins, outs = [], []
+    sets = input_sets(w)
+    xs, os_, ins, outs = [], [], [], []
     for s in range(sets):
         src = wl.Workload(w.name, N, count, block, w.dist, w.hidden, seed=w.seed + s)
         x = wl.make_inputs(src, device=dev)
-        ins.append([x[r] for r in range(N)])
         o = torch.empty_like(x)
+        xs.append(x)
+        os_.append(o)
+        ins.append([x[r] for r in range(N)])
         outs.append([o[r] for r in range(N)])
+    checksum = int(xs[0].view(torch.int16).to(torch.int64).bitwise_and(0xFFFF).sum().item())
     wb = eq.allreduce_sim_workspace_bytes(N, count, block, False)
     ws = torch.empty(wb, dtype=torch.uint8, device=dev)
     wbp = eq.allreduce_sim_pipelined_workspace_bytes(N, count, block, False)
     wsp = torch.empty(wbp, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream().cuda_stream
 
-    def step_pipelined(i):       # the headline: one deep-pipelined launch per step
+    def step_fused(i):           # the headline: the whole AllReduce as one chain-fused launch
         eq.allreduce_sim_pipelined(ins[i % sets], outs[i % sets], N, count, block, wsp, wbp, False, stream)
 
     def step_by_steps(i):        # one launch per ring step (N+1 launches)
@@ -303,53 +373,61 @@ def main():
     windows = []
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
-    def timed(step_fn, steps):
+    def timed(step_fn, steps, min_seconds=MIN_TIMED_SECONDS, max_trains=400):
+        """Trains of exactly `steps` steps between CUDA events on the launching stream, each bracketed
+        by a barrier + synchronize on both sides and reduced to the max over ranks; repeated until
+        min_seconds of GPU time has been measured.  Returns (median ms per step, trains)."""
         for i in range(args.warmup):
             step_fn(i)
-        barrier()
+        trains, total = [], 0.0
         h0 = time.perf_counter()
-        ev0.record()
-        for i in range(steps):
-            step_fn(i)
-        ev1.record()
-        torch.cuda.synchronize()
+        while len(trains) < 3 or (total < min_seconds * 1e3 and len(trains) < max_trains):
+            barrier()
+            ev0.record()
+            for i in range(steps):
+                step_fn(i)
+            ev1.record()
+            torch.cuda.synchronize()
+            barrier()
+            ms = max_over_ranks(ev0.elapsed_time(ev1), world, dev)
+            trains.append(ms)
+            total += ms
         windows.append((h0, time.perf_counter()))
-        barrier()
-        return max_over_ranks(ev0.elapsed_time(ev1), world, dev) / steps
+        return statistics.median(trains) / steps, len(trains)
 
     peak, peak_src = hbm_peak()
-    alg_bytes = algorithmic_bytes(N, count, block)
 
-    # ---- headline: the pipelined schedule; the timed region is exactly K launches of one kernel
-    ms_step = timed(step_pipelined, args.steps)
+    # ---- headline: the chain-fused single launch; a timed train is exactly K launches of one kernel
+    ms_step, trains = timed(step_fused, args.steps)
     value = aggregate_value(in_bytes, ms_step, world)
-    achieved = alg_bytes / (ms_step * 1e-3) / 1e9
-    traffic = PIPELINED_TRAFFIC_BYTES_PER_RANK_ELEMENT * count * N
-    roofline = {"bound": "hbm", "kernel": "pipelined_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
-                "algorithmic_bytes_per_launch": alg_bytes,
-                "dram_gbs": traffic / (ms_step * 1e-3) / 1e9, "dram_frac": traffic / (ms_step * 1e-3) / 1e9 / peak,
-                "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "note": "hop messages are written through to L2 and consumed at once from the SM's L1/L2, so DRAM "
-                        "traffic (inputs + outputs) is below the algorithmic bytes and frac can exceed 1"}
+    t = NCU_TRAFFIC["chain_fused_kernel"]
+    roofline = roofline_entry(
+        "chain_fused_kernel", chain_fused_bytes(N, count), ms_step, peak, peak_src,
+        t["bytes_per_element"] * count * N, f"ncu, {t['profile']}, scaled by elements",
+        "4*count*nranks: every bf16 input read once, every bf16 output written once; hop messages stay in registers")
+    roofline["ring_schedule_bytes_per_launch"] = ring_schedule_bytes(N, count, block)
+    roofline["note"] = ("frac counts only bytes this kernel moves through HBM; against the ring schedule's "
+                        "count*nranks*(6+8/block) bytes the same time would read "
+                        f"{ring_schedule_bytes(N, count, block) / (ms_step * 1e-3) / 1e9 / peak:.3f} of peak, "
+                        "which is not a fraction of anything this kernel does")
 
-    # ---- the same work as one launch per ring step
-    ms_steps = timed(step_by_steps, args.steps)
+    # ---- the same work as one launch per ring step: the hop messages go through memory
+    ms_steps, trains_steps = timed(step_by_steps, args.steps)
     # per-kernel durations: trains of launches between CUDA events, in stream order.  Launch 0
     # (quantize) and launch N (all-gather) are idempotent and are repeated 4 times per train so
     # that the events' own overhead is amortised; launches 1..N-1 (the hops) form one train.
-    trains = [("quantize_blocks", 0, 0, 4, 4)]
+    ktrains = [("quantize_blocks", 0, 0, 4, 4)]
     if N > 1:
-        trains.append(("rs_step_dequant_add_requant", 1, N - 1, 1, N - 1))
-    trains.append(("ag_dequant", N, N, 4, 4))
+        ktrains.append(("rs_step_dequant_add_requant", 1, N - 1, 1, N - 1))
+    ktrains.append(("ag_dequant", N, N, 4, 4))
     reps = max(5, min(50, args.steps))
-    evs = {t[0]: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-                  for _ in range(reps)] for t in trains}
+    evs = {t_[0]: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                   for _ in range(reps)] for t_ in ktrains}
     h0 = time.perf_counter()
     passes = 0
     while passes < 3 or (time.perf_counter() - h0 < 0.5 and passes < 2000):   # also gives the clock sampler load
         for i in range(reps):
-            for name, first, last, repeat, _ in trains:
+            for name, first, last, repeat, _ in ktrains:
                 a, b = evs[name][i]
                 a.record()
                 for _ in range(repeat):
@@ -360,9 +438,9 @@ def main():
         passes += 1
     windows.append((h0, time.perf_counter()))
     kernels = {}
-    train_ms = {t[0]: sum(a.elapsed_time(b) for a, b in evs[t[0]]) for t in trains}     # last pass
+    train_ms = {t_[0]: sum(a.elapsed_time(b) for a, b in evs[t_[0]]) for t_ in ktrains}     # last pass
     per_step_ms = {}
-    for name, first, last, repeat, launches in trains:
+    for name, first, last, repeat, launches in ktrains:
         avg_ms = train_ms[name] / (reps * launches)
         per_step = last - first + 1
         per_step_ms[name] = avg_ms * per_step
@@ -371,78 +449,91 @@ def main():
     for name in kernels:
         kernels[name]["share"] = per_step_ms[name] / sum(per_step_ms.values())
         kernels[name]["frac"] = kernels[name]["algorithmic_gbs"] / peak
-    steps_gbs = alg_bytes / (ms_steps * 1e-3) / 1e9
+    hop = NCU_TRAFFIC["rs_step_hop_small" if count * (1 + 4.0 / block) <= HOP_MESSAGES_STAY_IN_L2_BYTES
+                      else "rs_step_hop_large"]
     by_steps = {"value": aggregate_value(in_bytes, ms_steps, world), "unit": UNIT, "ms_per_step": ms_steps,
-                "gpu_launches_per_step": N + 1, "algorithmic_gbs": steps_gbs, "frac": steps_gbs / peak,
-                "frac_of_nominal_8TBs": steps_gbs / NOMINAL_HBM_GBS, "kernels": kernels,
-                "hop_traffic_bytes_per_launch": DAR_TRAFFIC_BYTES_PER_ELEMENT * count}
+                "trains": trains_steps, "gpu_launches_per_step": N + 1,
+                "roofline": roofline_entry(
+                    "rs_step_kernel x N + ag_dequant_kernel (whole step)", ring_schedule_bytes(N, count, block),
+                    ms_steps, peak, peak_src, None, "not captured for the whole step",
+                    "count*nranks*(6+8/block): N bf16 reads, every hop message written and read once, N bf16 writes"),
+                "kernels": kernels,
+                "hop_traffic_bytes_per_launch": hop["bytes_per_element"] * count,
+                "hop_traffic_source": f"ncu, {hop['profile']}, scaled by elements"}
 
-    # ---- the other flavours (semi-loop ring, stage selection), same workload, pipelined form
-    flavours = {}
-    wbf = eq.allreduce_sim_flavour_workspace_bytes(N, count, block, 7 if N % 2 == 0 else 6, False)
-    wsf = torch.empty(wbf, dtype=torch.uint8, device=dev)
-    names = {0: "full_loop_unquantized", 2: "full_loop_rs_only", 4: "full_loop_ag_only", 6: "full_loop_rs_ag",
-             1: "semi_loop_unquantized", 3: "semi_loop_rs_only", 5: "semi_loop_ag_only", 7: "semi_loop_rs_ag",
-             6 | 8: "full_loop_rs_ag_fp8_e4m3", 6 | 16: "full_loop_rs_ag_fp8_e5m2"}
-    for fl, name in sorted(names.items()):
-        if (fl & 1) and N % 2:
-            continue
-        ms_f = timed(lambda i, fl=fl: eq.allreduce_sim_flavour(ins[i % sets], outs[i % sets], N, count, block, fl,
-                                                               wsf, wbf, False, stream), max(5, min(200, args.steps)))
-        flavours[name] = {"ms_per_step": ms_f, "value": aggregate_value(in_bytes, ms_f, world), "unit": UNIT}
-    del wsf
+    flavours, bf16_sim, ratios = {}, None, None
+    if not args.no_extras:
+        # ---- the other flavours (semi-loop ring, stage selection, FP8), same workload, single launch
+        wbf = eq.allreduce_sim_flavour_workspace_bytes(N, count, block, 7 if N % 2 == 0 else 6, False)
+        wsf = torch.empty(wbf, dtype=torch.uint8, device=dev)
+        names = {0: "full_loop_unquantized", 2: "full_loop_rs_only", 4: "full_loop_ag_only", 6: "full_loop_rs_ag",
+                 1: "semi_loop_unquantized", 3: "semi_loop_rs_only", 5: "semi_loop_ag_only", 7: "semi_loop_rs_ag",
+                 6 | 8: "full_loop_rs_ag_fp8_e4m3", 6 | 16: "full_loop_rs_ag_fp8_e5m2"}
+        for fl, name in sorted(names.items()):
+            if (fl & 1) and N % 2:
+                continue
+            ms_f, _ = timed(lambda i, fl=fl: eq.allreduce_sim_flavour(ins[i % sets], outs[i % sets], N, count, block,
+                                                                      fl, wsf, wbf, False, stream),
+                            max(5, min(50, args.steps)), min_seconds=0.1)
+            flavours[name] = {"ms_per_step": ms_f, "value": aggregate_value(in_bytes, ms_f, world), "unit": UNIT}
+        del wsf
 
-    # unquantized comparator on the same GPU, same inputs
-    wb16 = eq.allreduce_sim_bf16_workspace_bytes(N, count)
-    ws16 = torch.empty(wb16, dtype=torch.uint8, device=dev)
-    for i in range(args.warmup):
-        eq.allreduce_sim_bf16(ins[i % sets], outs[i % sets], N, count, ws16, wb16, stream)
-    torch.cuda.synchronize()
-    h0 = time.perf_counter()
-    ev0.record()
-    for i in range(args.steps):
-        eq.allreduce_sim_bf16(ins[i % sets], outs[i % sets], N, count, ws16, wb16, stream)
-    ev1.record()
-    torch.cuda.synchronize()
-    windows.append((h0, time.perf_counter()))
-    ms16 = max_over_ranks(ev0.elapsed_time(ev1), world, dev) / args.steps
-    bf16_sim = {"value": in_bytes / (ms16 * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms16,
-                "algorithmic_bytes_per_step": count * (8 * N - 4),
-                "frac_of_measured_peak": count * (8 * N - 4) / (ms16 * 1e-3) / 1e9 / peak}
-    del ws16
+        # ---- unquantized comparator on the same GPU, same inputs, one launch per ring step
+        wb16 = eq.allreduce_sim_bf16_workspace_bytes(N, count)
+        ws16 = torch.empty(wb16, dtype=torch.uint8, device=dev)
+        ms16, _ = timed(lambda i: eq.allreduce_sim_bf16(ins[i % sets], outs[i % sets], N, count, ws16, wb16, stream),
+                        args.steps, min_seconds=0.2)
+        bf16_sim = {"value": aggregate_value(in_bytes, ms16, world), "unit": UNIT, "ms_per_step": ms16,
+                    "schedule": "one launch per ring step",
+                    "algorithmic_bytes_per_step": count * (8 * N - 4),
+                    "frac_of_measured_peak": count * (8 * N - 4) / (ms16 * 1e-3) / 1e9 / peak}
+        del ws16
+        # like for like: the same schedule form on both sides of each ratio
+        ratios = {"single_launch_quantized_over_single_launch_bf16":
+                      flavours["full_loop_unquantized"]["ms_per_step"] / ms_step,
+                  "per_step_quantized_over_per_step_bf16": ms16 / ms_steps}
 
-    # end to end through the host-buffer front end: every step uploads its N input tensors from
-    # pinned host memory, runs the AllReduce and downloads the N outputs; copies of neighbouring
-    # steps overlap with the kernels (three streams, two device buffer sets)
+    # ---- end to end through the C ABI's host-buffer entry: every step uploads its N input tensors
+    # from pinned host memory, reduces them and downloads the N outputs.  Two streams and two staging
+    # buffers, used alternately, so that one step's upload overlaps the previous step's download.
     e2e = None
     if not args.no_e2e:
-        from paper_2506_17615_b200.host_api import HostPipeline
         h_in = [torch.empty((N, count), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
         for i, h in enumerate(h_in):
-            h.copy_(torch.stack(ins[i % sets]).cpu())
+            h.copy_(xs[i % sets])
         h_out = [torch.empty((N, count), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
-        pipe = HostPipeline(N, count, block, dev)
-        e_steps = max(3, min(20, args.steps))
+        sb = eq.allreduce_sim_host_staging_bytes(N, count)
+        stage = [torch.empty(sb, dtype=torch.uint8, device=dev) for _ in range(2)]
+        side = [torch.cuda.Stream(dev) for _ in range(2)]
+
+        def host_step(i):
+            eq.allreduce_sim_host([h_in[i % 2][r] for r in range(N)], [h_out[i % 2][r] for r in range(N)], N, count,
+                                  block, stage[i % 2], sb, side[i % 2].cuda_stream)
+
+        e_steps = max(3, min(10, args.steps))
         for i in range(3):
-            pipe.submit(h_in[i % 2], h_out[i % 2])
-        pipe.wait()
+            host_step(i)
         barrier()
         t0 = torch.cuda.Event(enable_timing=True)
         t1 = torch.cuda.Event(enable_timing=True)
-        t0.record()
-        pipe.h2d.wait_event(t0)
+        cur = torch.cuda.current_stream()
+        h0 = time.perf_counter()
+        t0.record(cur)
+        for s_ in side:
+            s_.wait_event(t0)
         for i in range(e_steps):
-            pipe.submit(h_in[i % 2], h_out[i % 2])
-        torch.cuda.current_stream().wait_stream(pipe.d2h)
-        torch.cuda.current_stream().wait_stream(pipe.comp)
-        t1.record()
+            host_step(i)
+        for s_ in side:
+            cur.wait_stream(s_)
+        t1.record(cur)
         torch.cuda.synchronize()
+        windows.append((h0, time.perf_counter()))
         barrier()
         ms_e = max_over_ranks(t0.elapsed_time(t1), world, dev) / e_steps
         e2e = {"value": aggregate_value(in_bytes, ms_e, world), "unit": UNIT, "h2d_bytes_per_step": in_bytes,
                "d2h_bytes_per_step": in_bytes, "ms_per_step": ms_e, "steps": e_steps,
-               "api": "paper_2506_17615_b200.host_api.HostPipeline.submit (copies overlapped across steps)"}
-        del h_in, h_out, pipe
+               "api": "equarx_allreduce_sim_host (C ABI, host pointers); two streams and staging buffers in rotation"}
+        del h_in, h_out, stage
 
     sampler.stop()
     clocks = sampler.summary(windows)
@@ -450,19 +541,22 @@ def main():
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {**base_config(w), "parallelism": f"replicas x{world}" if world > 1 else "1 GPU",
-                       "l2": f"{sets} input/output sets used in rotation ({sets * 2 * in_bytes / 1e6:.0f} MB "
-                             f"working set against a 126 MB L2); no explicit flush",
-                       "pdl_between_step_launches": os.environ.get("EQUARX_PDL", "1") != "0"},
+            "warmup": args.warmup, "ms_per_step": ms_step, "trains": trains, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": base_config(w, world),
             "e2e": e2e, "gpu_launches": args.steps, "clocks": clocks,
-            "roofline": roofline, "schedule": "pipelined (equarx_allreduce_sim_pipelined, 1 launch per step)",
+            "roofline": roofline,
+            "schedule": "chain-fused single launch (equarx_allreduce_sim_pipelined, keep_trace=0)",
             "by_steps": by_steps, "flavours": flavours, "bf16_sim": bf16_sim,
-            "speedup_vs_bf16_sim": value / world / bf16_sim["value"],
+            "speedup_vs_bf16": ratios, "input_checksum": checksum,
+            "pdl_between_step_launches": os.environ.get("EQUARX_PDL", "1") != "0",
         }
         if world == 1 and not args.no_cpu_baseline:
-            line["cpu_baseline"] = cpu_baseline(w)
+            # the outputs of the last chain-fused step on set 0 are recomputed so that the parity verdict
+            # belongs to the kernel that was timed
+            step_fused(0)
+            torch.cuda.synchronize()
+            line["cpu_baseline"], line["parity"] = cpu_baseline_and_parity(w, xs[0], os_[0])
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -71,9 +71,10 @@ enum equarx_status {
 };
 
 /*
- * Ring step 0 (Section 3.1: "quantize the shard, send the quantized shard and
- * the corresponding metadata"; two phases Q_p1 = metadata, Q_p2 = scaling,
- * fused here into one pass over registers).
+ * Ring step 0 (Section 3.1): the shard a rank sends first is quantized; what
+ * travels is the int8 payload together with its scale factors.  The paper's two
+ * phases (Q_p1 finds the metadata, Q_p2 scales the data) are one pass over
+ * registers here.
  *   x_bf16 : count bf16 words (device, read)
  *   codes  : count int8 (device, written)
  *   scales : count/block fp32 (device, written); scales[b] belongs to
@@ -84,9 +85,9 @@ int equarx_quantize_blocks(const void *x_bf16, size_t count, int block,
                            int8_t *codes, float *scales, equarx_stream_t stream);
 
 /*
- * Ring steps 1..N-1 (Section 3.1: "dequantize the received shard to higher
- * precision (e.g. FP32), and perform the addition", then quantize the partial
- * sum for the next hop).  The fp32 partial sum lives in registers only.
+ * Ring steps 1..N-1 (Section 3.1): the received shard is widened to fp32 and
+ * added to this rank's counterpart, and the partial sum is quantized again for
+ * the next hop.  The fp32 partial sum lives in registers only.
  *   codes_in, scales_in   : the received message (device, read)
  *   local_bf16            : this rank's counterpart shard, count bf16 (device, read)
  *   codes_out, scales_out : the message for the next hop (device, written);
@@ -112,7 +113,7 @@ int equarx_ag_dequant(const int8_t *codes, const float *scales, size_t count, in
  * scales) is stored as a sequence of 544-byte records, one per tile of 512
  * consecutive elements of the shard: first 8 floats of metadata (the tile's
  * 512/block scales in order, then zeros), then the tile's 512 int8 codes
- * ("send the metadata before any microshards", Section 3.1).  The last record
+ * (metadata ahead of the payload it describes, the order Section 3.1 sends them in).  The last record
  * of a message is only partly used if the shard is not a multiple of 512.
  * A message slot is tiles = ceil(shard/512) records; slot i starts at byte
  * i*tiles*544.  "Event j of shard k" is the message sent at ring step j by rank
@@ -162,24 +163,32 @@ int equarx_allreduce_sim_range(const void *const *in_bf16, void *const *out_bf16
                                int first_launch, int last_launch, equarx_stream_t stream);
 
 /*
- * The same AllReduce as ONE persistent launch in deep-pipelined order.  Section
- * 3.1 splits a shard into microshards that move through the ring steps
- * independently of one another; here a microshard is a tile of 512 elements
- * and one warp carries it through all nranks steps and the all-gather without
- * waiting for the rest of the shard.  Every hop message is still written to
- * memory as a record and read back from there (by the neighbouring lane, acting
- * for the receiving rank), but it is consumed right after it was produced and is
- * therefore served from the SM's L1/L2 instead of HBM.  Outputs, and with keep_trace the
- * whole trace, are identical to equarx_allreduce_sim bit for bit; only the order
- * in which tiles advance differs.
+ * The same AllReduce as ONE persistent launch.  Section 3.1 splits a shard into
+ * microshards that move through the ring steps independently of one another;
+ * here a microshard is a tile of 512 elements and one warp carries it through
+ * all nranks steps and the all-gather without waiting for the rest of the
+ * shard.  Outputs, and with keep_trace the whole trace, are identical to
+ * equarx_allreduce_sim bit for bit; only the order in which tiles advance
+ * differs.  Two forms:
  *
- * Workspace: with keep_trace, the trace exactly as equarx_allreduce_sim lays it
- * out.  Without, EQUARX_PIPELINE_FIFO_BYTES of staging space: every warp owns a
- * two-record FIFO that it reuses for all steps of all its tiles (the way a ring
- * channel reuses its staging buffers); its contents on return are meaningless.
+ *   keep_trace != 0 (deep-pipelined, every message materialised): each hop
+ *     message is written to memory as a record and read back from there by the
+ *     neighbouring lane, which acts for the receiving rank.  The workspace
+ *     receives the trace exactly as equarx_allreduce_sim lays it out.
+ *   keep_trace == 0 (chain-fused): the adder chain of a tile (Section 3.3,
+ *     Fig. 4) depends on no other tile, so the lane that quantized a group for
+ *     the sending rank continues as the receiving rank; the message (int8 code
+ *     values and the block scale) stays in registers and is never stored.  The
+ *     kernel reads every bf16 input once and writes every bf16 output once:
+ *     4 bytes of memory traffic per element of every rank, which is the
+ *     roofline of this form; the hop messages of the ring schedule
+ *     (2 + 8/block more bytes per element) are not moved at all.  The workspace
+ *     is not touched; EQUARX_PIPELINE_MIN_WORKSPACE_BYTES is a token size so that
+ *     one allocation pattern serves both forms.
+ *
  * All other arguments and rules as for equarx_allreduce_sim.
  */
-#define EQUARX_PIPELINE_FIFO_BYTES (8u * 1024u * 1024u)
+#define EQUARX_PIPELINE_MIN_WORKSPACE_BYTES 32u
 size_t equarx_allreduce_sim_pipelined_workspace_bytes(int nranks, size_t count, int block, int keep_trace);
 int equarx_allreduce_sim_pipelined(const void *const *in_bf16, void *const *out_bf16,
                                    int nranks, size_t count, int block,
@@ -187,10 +196,35 @@ int equarx_allreduce_sim_pipelined(const void *const *in_bf16, void *const *out_
                                    equarx_stream_t stream);
 
 /*
+ * The AllReduce of equarx_allreduce_sim_pipelined (keep_trace = 0) for tensors
+ * that live in HOST memory: what Section 3.1 and Section 3.4 compute, with the
+ * copies to and from the device issued by this call.
+ *   host_in[r]  : count bf16 words of rank r in host memory (read).  Pinned
+ *                 (page-locked) memory makes the copies asynchronous; pageable
+ *                 memory works and makes the call block for the copies.
+ *   host_out[r] : count bf16 words in host memory (written); may equal
+ *                 host_in[r].
+ *   staging     : DEVICE memory supplied by the caller,
+ *                 equarx_allreduce_sim_host_staging_bytes(nranks, count) bytes
+ *                 (2 * count * nranks), 32-byte aligned; holds the nranks
+ *                 tensors on the device and is reduced in place.
+ * The call enqueues on `stream`: nranks host-to-device copies (one plain
+ * cudaMemcpyAsync per rank tensor), the kernel, nranks device-to-host copies, and
+ * returns without synchronising; host_out is valid once the stream has reached the
+ * last copy.  The library still allocates nothing.  A failing copy is reported as
+ * EQUARX_ERR_CUDA like a failing launch.  Two calls on two streams with two
+ * staging buffers overlap each other's copies and kernels.
+ */
+size_t equarx_allreduce_sim_host_staging_bytes(int nranks, size_t count);
+int equarx_allreduce_sim_host(const void *const *host_in, void *const *host_out,
+                              int nranks, size_t count, int block,
+                              void *staging, size_t staging_bytes,
+                              equarx_stream_t stream);
+
+/*
  * The other flavours of the method, in the deep-pipelined form of
  * equarx_allreduce_sim_pipelined (one persistent launch, one warp per
- * 512-element tile, every message through the warp's staging FIFO and read
- * back by the neighbouring lane).  `flavour` is a combination of:
+ * 512-element tile).  `flavour` is a combination of:
  *   EQUARX_FLAVOUR_SEMI_LOOP : semi-loop ring (Section 3.3, Fig. 5): shard k is
  *       reduced by two half chains that meet at its owner,
  *       A: k+N/2 -> k+N/2-1 -> ... -> k+1 -> k and B: k+N/2+1 -> ... -> k-1 -> k
@@ -213,11 +247,16 @@ int equarx_allreduce_sim_pipelined(const void *const *in_bf16, void *const *out_
  *       as -0.0.  The codes of a trace are the raw FP8 bytes.
  * QUANT_RS | QUANT_AG is equarx_allreduce_sim_pipelined's result bit for bit;
  * 0 is the unquantized ring of equarx_allreduce_sim_bf16.
- * Workspace: EQUARX_FLAVOUR_FIFO_BYTES of staging space, followed, with
- * keep_trace, by a trace laid out as for equarx_allreduce_sim.  Events of a
- * full loop: j = 0..N-2 the hops in chain order, N-1 the all-gather message;
- * of a semi loop: 0..N/2-1 chain A's hops, N/2..N-2 chain B's hops, N-1 the
- * all-gather message.  Events that the flavour does not quantize are zeroed.
+ * Like equarx_allreduce_sim_pipelined the call has two forms.  Without
+ * keep_trace every message stays in the registers of the lane that produced it
+ * (chain-fused; for flavour 0 this is the unquantized comparator in the same
+ * form as the quantized single launch) and the workspace, of the token size
+ * EQUARX_PIPELINE_MIN_WORKSPACE_BYTES, is not touched.  With keep_trace every
+ * message goes through memory and the workspace is EQUARX_FLAVOUR_FIFO_BYTES of
+ * staging space followed by a trace laid out as for equarx_allreduce_sim.
+ * Events of a full loop: j = 0..N-2 the hops in chain order, N-1 the all-gather
+ * message; of a semi loop: 0..N/2-1 chain A's hops, N/2..N-2 chain B's hops, N-1
+ * the all-gather message.  Events that the flavour does not quantize are zeroed.
  * Other arguments and rules as for equarx_allreduce_sim.
  */
 #define EQUARX_FLAVOUR_SEMI_LOOP 1

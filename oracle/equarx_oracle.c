@@ -18,8 +18,8 @@
  * adds the local counterpart, requantizes and forwards; the all-gather
  * forwards the last message and everybody dequantizes it).  There is no
  * blocking, fusion or reordering beyond that.  Precision is the paper's:
- * bf16 tensors, int8 payload, fp32 accumulation ("higher precision (e.g.
- * FP32)", Section 3.1).  Where the paper is silent the reading taken is
+ * bf16 tensors, int8 payload, fp32 accumulation (Section 3.1 widens the
+ * received shard before adding and names FP32).  Where the paper is silent the reading taken is
  * stated next to the code:
  *   - ring direction: rank r sends to rank (r+1) mod N; shard k ends on
  *     rank k (the semi-loop example of Section 3.3 finishes shard 0 on

@@ -29,7 +29,13 @@ def is_stale():
 
 
 def build(force=False, verbose=False):
-    """Compile libequarx.so next to this file; returns its path."""
+    """Compile libequarx.so next to this file; returns its path.  EQUARX_LIBRARY=<path> in the
+    environment selects an already built library instead (nothing is compiled then)."""
+    prebuilt = os.environ.get("EQUARX_LIBRARY")
+    if prebuilt and not force:
+        if not os.path.exists(prebuilt):
+            raise RuntimeError(f"EQUARX_LIBRARY={prebuilt} does not exist")
+        return prebuilt
     if not force and not is_stale():
         return LIB
     nvcc = find_nvcc()

@@ -26,6 +26,8 @@ EXPORTS = (
     "equarx_allreduce_sim_flavour_workspace_bytes",
     "equarx_allreduce_sim_pipelined",
     "equarx_allreduce_sim_pipelined_workspace_bytes",
+    "equarx_allreduce_sim_host",
+    "equarx_allreduce_sim_host_staging_bytes",
     "equarx_allreduce_sim_range",
     "equarx_allreduce_sim_static",
     "equarx_allreduce_sim_bf16_workspace_bytes",
@@ -55,6 +57,9 @@ def _load():
     lib.equarx_allreduce_sim_pipelined.argtypes = [vp, vp, ci, sz, ci, vp, sz, ci, vp]
     lib.equarx_allreduce_sim_pipelined_workspace_bytes.argtypes = [ci, sz, ci, ci]
     lib.equarx_allreduce_sim_pipelined_workspace_bytes.restype = sz
+    lib.equarx_allreduce_sim_host.argtypes = [vp, vp, ci, sz, ci, vp, sz, vp]
+    lib.equarx_allreduce_sim_host_staging_bytes.argtypes = [ci, sz]
+    lib.equarx_allreduce_sim_host_staging_bytes.restype = sz
     lib.equarx_allreduce_sim_flavour.argtypes = [vp, vp, ci, sz, ci, ci, vp, sz, ci, vp]
     lib.equarx_allreduce_sim_flavour_workspace_bytes.argtypes = [ci, sz, ci, ci, ci]
     lib.equarx_allreduce_sim_flavour_workspace_bytes.restype = sz
@@ -72,7 +77,7 @@ def _load():
 
 
 lib = _load()
-LIB_PATH = _build.LIB
+LIB_PATH = lib._name
 
 
 def _ptr(x):
@@ -139,6 +144,18 @@ def allreduce_sim_pipelined(in_bf16, out_bf16, nranks, count, block, workspace, 
            "equarx_allreduce_sim_pipelined")
 
 
+def allreduce_sim_host_staging_bytes(nranks, count):
+    return lib.equarx_allreduce_sim_host_staging_bytes(nranks, count)
+
+
+def allreduce_sim_host(host_in, host_out, nranks, count, block, staging, staging_bytes, stream=0):
+    """equarx_allreduce_sim_host: host_in / host_out are HOST pointers (integers, or pinned CPU
+    tensors with data_ptr()), staging is device memory; copies and kernel go to `stream`."""
+    _check(lib.equarx_allreduce_sim_host(_table(host_in), _table(host_out), nranks, count, block, _ptr(staging),
+                                         staging_bytes, _ptr(stream)),
+           "equarx_allreduce_sim_host")
+
+
 def allreduce_sim_flavour_workspace_bytes(nranks, count, block, flavour, keep_trace=False):
     return lib.equarx_allreduce_sim_flavour_workspace_bytes(nranks, count, block, flavour, int(bool(keep_trace)))
 
@@ -178,7 +195,7 @@ def allreduce_sim_bf16(in_bf16, out_bf16, nranks, count, workspace, workspace_by
 
 
 RECORD_BYTES, RECORD_HEADER, TILE_ELEMS = 544, 32, 512
-PIPELINE_FIFO_BYTES = 8 * 1024 * 1024
+PIPELINE_MIN_WORKSPACE_BYTES = 32
 
 
 def trace_views(workspace_u8, nranks, count, block, keep_trace=True):

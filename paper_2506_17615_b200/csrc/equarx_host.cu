@@ -5,6 +5,7 @@
 #include "equarx_kernels.cuh"
 
 #include <algorithm>
+#include <atomic>
 #include <cstdlib>
 #include <cstring>
 
@@ -159,6 +160,28 @@ const void* flavour_kernel_for(int flavour) {
     if (flavour & EQUARX_FLAVOUR_E4M3) return flavour_kernel_for<LPB, 2>(flavour);
     if (flavour & EQUARX_FLAVOUR_E5M2) return flavour_kernel_for<LPB, 3>(flavour);
     return flavour_kernel_for<LPB, 1>(flavour);
+}
+
+// the same flavours with the messages kept in registers (no trace)
+template <int LPB, int PAYLOAD>
+const void* flavour_fused_kernel_for(int flavour) {
+    switch (flavour & 7) {
+        case 2: return reinterpret_cast<const void*>(flavour_fused_kernel<LPB, false, true, false, PAYLOAD>);
+        case 3: return reinterpret_cast<const void*>(flavour_fused_kernel<LPB, true, true, false, PAYLOAD>);
+        case 4: return reinterpret_cast<const void*>(flavour_fused_kernel<LPB, false, false, true, PAYLOAD>);
+        case 5: return reinterpret_cast<const void*>(flavour_fused_kernel<LPB, true, false, true, PAYLOAD>);
+        case 6: return reinterpret_cast<const void*>(flavour_fused_kernel<LPB, false, true, true, PAYLOAD>);
+        case 7: return reinterpret_cast<const void*>(flavour_fused_kernel<LPB, true, true, true, PAYLOAD>);
+        case 1: return reinterpret_cast<const void*>(flavour_fused_kernel<LPB, true, false, false, 1>);
+        default: return reinterpret_cast<const void*>(flavour_fused_kernel<LPB, false, false, false, 1>);
+    }
+}
+
+template <int LPB>
+const void* flavour_fused_kernel_for(int flavour) {
+    if (flavour & EQUARX_FLAVOUR_E4M3) return flavour_fused_kernel_for<LPB, 2>(flavour);
+    if (flavour & EQUARX_FLAVOUR_E5M2) return flavour_fused_kernel_for<LPB, 3>(flavour);
+    return flavour_fused_kernel_for<LPB, 1>(flavour);
 }
 
 // a valid flavour: any of the three schedule bits, at most one payload bit, and a payload bit
@@ -325,19 +348,15 @@ int equarx_allreduce_sim_range(const void* const* in_bf16, void* const* out_bf16
 size_t equarx_allreduce_sim_pipelined_workspace_bytes(int nranks, size_t count, int block, int keep_trace) {
     if (check_sim_shape(nranks, count, block) != EQUARX_OK) return 0;
     if (keep_trace) return equarx_allreduce_sim_workspace_bytes(nranks, count, block, 1);
-    return size_t(EQUARX_PIPELINE_FIFO_BYTES);
+    return size_t(EQUARX_PIPELINE_MIN_WORKSPACE_BYTES);      // not touched: the chain-fused kernel needs no scratch
 }
 
-int equarx_allreduce_sim_pipelined(const void* const* in_bf16, void* const* out_bf16, int nranks, size_t count,
-                                   int block, void* workspace, size_t workspace_bytes, int keep_trace,
-                                   equarx_stream_t stream) {
-    if (int st = check_sim_shape(nranks, count, block)) return st;
-    if (!workspace) return EQUARX_ERR_NULL;
-    const size_t need = equarx_allreduce_sim_pipelined_workspace_bytes(nranks, count, block, keep_trace);
-    if (workspace_bytes < need) return EQUARX_ERR_WORKSPACE;
-    if (!aligned(workspace, 32)) return EQUARX_ERR_ALIGN;
-    if (int st = check_tables(in_bf16, out_bf16, nranks, 2 * count, workspace, need)) return st;
+}  // extern "C"
 
+namespace {
+// the single-launch schedule on validated arguments (workspace: the trace, or unused)
+int launch_pipelined(const void* const* in_bf16, void* const* out_bf16, int nranks, size_t count, int block,
+                     void* workspace, int keep_trace, cudaStream_t stream, bool quantized = true) {
     const uint32_t N = uint32_t(nranks);
     const size_t shard = count / N;
     PipeArgs a = {};
@@ -350,19 +369,20 @@ int equarx_allreduce_sim_pipelined(const void* const* in_bf16, void* const* out_
     a.shard = shard;
     a.tiles_per_shard = (shard + kTileElems - 1) / kTileElems;
     a.nranks = N;
-    a.keep_trace = keep_trace ? 1u : 0u;
 
+    constexpr int D = EQX_FUSED_DEPTH;
     const void* kernel = nullptr;
+#define EQX_PICK(L)                                                                                   \
+    kernel = keep_trace ? reinterpret_cast<const void*>(pipelined_kernel<L>)                          \
+             : quantized ? reinterpret_cast<const void*>(chain_fused_kernel<L, D, true>)              \
+                         : reinterpret_cast<const void*>(chain_fused_kernel<L, D, false>)
     switch (block) {
-        case 64: kernel = keep_trace ? reinterpret_cast<const void*>(pipelined_kernel<4, true>)
-                                     : reinterpret_cast<const void*>(pipelined_kernel<4, false>); break;
-        case 128: kernel = keep_trace ? reinterpret_cast<const void*>(pipelined_kernel<8, true>)
-                                      : reinterpret_cast<const void*>(pipelined_kernel<8, false>); break;
-        case 256: kernel = keep_trace ? reinterpret_cast<const void*>(pipelined_kernel<16, true>)
-                                      : reinterpret_cast<const void*>(pipelined_kernel<16, false>); break;
-        default: kernel = keep_trace ? reinterpret_cast<const void*>(pipelined_kernel<32, true>)
-                                     : reinterpret_cast<const void*>(pipelined_kernel<32, false>); break;
+        case 64: EQX_PICK(4); break;
+        case 128: EQX_PICK(8); break;
+        case 256: EQX_PICK(16); break;
+        default: EQX_PICK(32); break;
     }
+#undef EQX_PICK
     // persistent grid: a whole number of CTAs per SM
     int dev = 0, sms = 0, occ = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -388,9 +408,6 @@ int equarx_allreduce_sim_pipelined(const void* const* in_bf16, void* const* out_
     }
     const uint64_t max_needed = (tiles + wpc - 1) / wpc;
     if (best_ctas > max_needed) best_ctas = max_needed;
-    // every warp owns a two-record staging FIFO in the workspace
-    const uint64_t fifo_ctas = uint64_t(EQUARX_PIPELINE_FIFO_BYTES) / (2 * kRecordBytes) / wpc;
-    if (!keep_trace && best_ctas > fifo_ctas) best_ctas = fifo_ctas;
 
     // programmatic dependent launch hides the launch latency behind the previous kernel's tail; the
     // kernel itself waits for that kernel to complete before its first memory access
@@ -413,15 +430,75 @@ int equarx_allreduce_sim_pipelined(const void* const* in_bf16, void* const* out_
     }
     return EQUARX_OK;
 }
+}  // namespace
+
+extern "C" {
+
+int equarx_allreduce_sim_pipelined(const void* const* in_bf16, void* const* out_bf16, int nranks, size_t count,
+                                   int block, void* workspace, size_t workspace_bytes, int keep_trace,
+                                   equarx_stream_t stream) {
+    if (int st = check_sim_shape(nranks, count, block)) return st;
+    if (!workspace) return EQUARX_ERR_NULL;
+    const size_t need = equarx_allreduce_sim_pipelined_workspace_bytes(nranks, count, block, keep_trace);
+    if (workspace_bytes < need) return EQUARX_ERR_WORKSPACE;
+    if (!aligned(workspace, 32)) return EQUARX_ERR_ALIGN;
+    if (int st = check_tables(in_bf16, out_bf16, nranks, 2 * count, workspace, need)) return st;
+    return launch_pipelined(in_bf16, out_bf16, nranks, count, block, workspace, keep_trace, stream);
+}
+
+size_t equarx_allreduce_sim_host_staging_bytes(int nranks, size_t count) {
+    if (nranks < 1 || nranks > EQUARX_MAX_RANKS || count == 0 || count > kMaxCount) return 0;
+    return 2 * count * size_t(nranks);
+}
+
+int equarx_allreduce_sim_host(const void* const* host_in, void* const* host_out, int nranks, size_t count,
+                              int block, void* staging, size_t staging_bytes, equarx_stream_t stream) {
+    if (int st = check_sim_shape(nranks, count, block)) return st;
+    if (!host_in || !host_out || !staging) return EQUARX_ERR_NULL;
+    for (int r = 0; r < nranks; ++r)
+        if (!host_in[r] || !host_out[r]) return EQUARX_ERR_NULL;
+    const size_t bytes = 2 * count;
+    if (staging_bytes < bytes * size_t(nranks)) return EQUARX_ERR_WORKSPACE;
+    if (!aligned(staging, 32)) return EQUARX_ERR_ALIGN;
+    for (int r = 0; r < nranks; ++r) {
+        if (!aligned(host_in[r], 2) || !aligned(host_out[r], 2)) return EQUARX_ERR_ALIGN;
+        for (int q = 0; q < nranks; ++q) {
+            if (q != r && overlap(host_out[r], bytes, host_out[q], bytes)) return EQUARX_ERR_ALIAS;
+            if (overlap(host_out[r], bytes, host_in[q], bytes) && !(q == r && host_out[r] == host_in[r]))
+                return EQUARX_ERR_ALIAS;
+        }
+    }
+    const void* dev_in[EQUARX_MAX_RANKS];
+    void* dev_out[EQUARX_MAX_RANKS];
+    for (int r = 0; r < nranks; ++r) dev_in[r] = dev_out[r] = static_cast<char*>(staging) + size_t(r) * bytes;
+
+    auto failed = [](cudaError_t e) {
+        g_last_cuda_error = int(e);
+        (void)cudaGetLastError();
+        return EQUARX_ERR_CUDA;
+    };
+    cudaError_t e = injected_launch_error();
+    if (e != cudaSuccess) return failed(e);
+    for (int r = 0; r < nranks; ++r) {
+        e = cudaMemcpyAsync(dev_out[r], host_in[r], bytes, cudaMemcpyHostToDevice, stream);
+        if (e != cudaSuccess) return failed(e);
+    }
+    // reduced in place in the staging buffer; the chain-fused kernel needs no workspace
+    if (int st = launch_pipelined(dev_in, dev_out, nranks, count, block, nullptr, 0, stream)) return st;
+    for (int r = 0; r < nranks; ++r) {
+        e = cudaMemcpyAsync(host_out[r], dev_out[r], bytes, cudaMemcpyDeviceToHost, stream);
+        if (e != cudaSuccess) return failed(e);
+    }
+    return EQUARX_OK;
+}
 
 size_t equarx_allreduce_sim_flavour_workspace_bytes(int nranks, size_t count, int block, int flavour,
                                                     int keep_trace) {
     if (check_sim_shape(nranks, count, block) != EQUARX_OK) return 0;
     if (!flavour_ok(flavour)) return 0;
     if ((flavour & EQUARX_FLAVOUR_SEMI_LOOP) && nranks % 2 != 0) return 0;
-    size_t bytes = size_t(EQUARX_FLAVOUR_FIFO_BYTES);
-    if (keep_trace) bytes += equarx_allreduce_sim_workspace_bytes(nranks, count, block, 1);
-    return bytes;
+    if (!keep_trace) return size_t(EQUARX_PIPELINE_MIN_WORKSPACE_BYTES);   // messages stay in registers
+    return size_t(EQUARX_FLAVOUR_FIFO_BYTES) + equarx_allreduce_sim_workspace_bytes(nranks, count, block, 1);
 }
 
 int equarx_allreduce_sim_flavour(const void* const* in_bf16, void* const* out_bf16, int nranks, size_t count,
@@ -438,13 +515,20 @@ int equarx_allreduce_sim_flavour(const void* const* in_bf16, void* const* out_bf
 
     const uint32_t N = uint32_t(nranks);
     const size_t shard = count / N;
+    if (!keep_trace) {
+        // the full loop with both stages quantized (int8) and the unquantized full loop have the tuned kernel
+        const int sched = flavour & 7;
+        const bool fp8 = flavour & (EQUARX_FLAVOUR_E4M3 | EQUARX_FLAVOUR_E5M2);
+        if (sched == 0 || (sched == (EQUARX_FLAVOUR_QUANT_RS | EQUARX_FLAVOUR_QUANT_AG) && !fp8))
+            return launch_pipelined(in_bf16, out_bf16, nranks, count, block, nullptr, 0, stream, sched != 0);
+    }
     FlavourArgs a = {};
     a.neg_zero = -0.0f;
     for (uint32_t r = 0; r < N; ++r) {
         a.in[r] = in_bf16[r];
         a.out[r] = out_bf16[r];
     }
-    a.fifo = static_cast<char*>(workspace);
+    a.fifo = keep_trace ? static_cast<char*>(workspace) : nullptr;
     a.trace = keep_trace ? static_cast<char*>(workspace) + size_t(EQUARX_FLAVOUR_FIFO_BYTES) : nullptr;
     a.shard = shard;
     a.tiles_per_shard = (shard + kTileElems - 1) / kTileElems;
@@ -452,10 +536,10 @@ int equarx_allreduce_sim_flavour(const void* const* in_bf16, void* const* out_bf
 
     const void* kernel = nullptr;
     switch (block) {
-        case 64: kernel = flavour_kernel_for<4>(flavour); break;
-        case 128: kernel = flavour_kernel_for<8>(flavour); break;
-        case 256: kernel = flavour_kernel_for<16>(flavour); break;
-        default: kernel = flavour_kernel_for<32>(flavour); break;
+        case 64: kernel = keep_trace ? flavour_kernel_for<4>(flavour) : flavour_fused_kernel_for<4>(flavour); break;
+        case 128: kernel = keep_trace ? flavour_kernel_for<8>(flavour) : flavour_fused_kernel_for<8>(flavour); break;
+        case 256: kernel = keep_trace ? flavour_kernel_for<16>(flavour) : flavour_fused_kernel_for<16>(flavour); break;
+        default: kernel = keep_trace ? flavour_kernel_for<32>(flavour) : flavour_fused_kernel_for<32>(flavour); break;
     }
     int dev = 0, sms = 0, occ = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -476,7 +560,7 @@ int equarx_allreduce_sim_flavour(const void* const* in_bf16, void* const* out_bf
         }
     }
     ctas = std::min<uint64_t>(ctas, (tiles + wpc - 1) / wpc);
-    ctas = std::min<uint64_t>(ctas, uint64_t(EQUARX_FLAVOUR_FIFO_BYTES) / (2 * kFifoEntryBytes) / wpc);
+    if (keep_trace) ctas = std::min<uint64_t>(ctas, uint64_t(EQUARX_FLAVOUR_FIFO_BYTES) / (2 * kFifoEntryBytes) / wpc);
     if (keep_trace) {                                  // events that this flavour does not quantize stay zero
         e = cudaMemsetAsync(a.trace, 0, need - size_t(EQUARX_FLAVOUR_FIFO_BYTES), stream);
         if (e != cudaSuccess) {
@@ -553,31 +637,37 @@ static __device__ __align__(256) unsigned char g_static_workspace[EQUARX_STATIC_
 
 namespace {
 constexpr int kMaxDevices = 64;
-void* g_static_ptr[kMaxDevices] = {};      // device address of g_static_workspace, per device ordinal
+// device address of g_static_workspace, per device ordinal (every thread that sets it stores the same value)
+std::atomic<void*> g_static_ptr[kMaxDevices];
 }  // namespace
 
 int equarx_allreduce_sim_static(const void* const* in_bf16, void* const* out_bf16, int nranks, size_t count,
                                 int block, equarx_stream_t stream) {
+    // host-side validation first: no CUDA call is made for arguments that are rejected
     if (int st = check_sim_shape(nranks, count, block)) return st;
     const size_t need = equarx_allreduce_sim_workspace_bytes(nranks, count, block, 0);
     if (need > size_t(EQUARX_STATIC_WORKSPACE_BYTES)) return EQUARX_ERR_STATIC_LIMIT;
+    if (int st = check_tables(in_bf16, out_bf16, nranks, 2 * count, nullptr, 0)) return st;
 
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess && (dev < 0 || dev >= kMaxDevices)) e = cudaErrorInvalidDevice;
-    if (e == cudaSuccess && g_static_ptr[dev] == nullptr) {
-        // set-up, once per device, with that device current (a benign race: every
-        // thread that gets here stores the same address)
-        void* p = nullptr;
-        e = cudaGetSymbolAddress(&p, g_static_workspace);
-        if (e == cudaSuccess) g_static_ptr[dev] = p;
+    void* ws = nullptr;
+    if (e == cudaSuccess) {
+        ws = g_static_ptr[dev].load(std::memory_order_relaxed);
+        if (ws == nullptr) {
+            // set-up, once per device, with that device current
+            e = cudaGetSymbolAddress(&ws, g_static_workspace);
+            if (e == cudaSuccess) g_static_ptr[dev].store(ws, std::memory_order_relaxed);
+        }
     }
     if (e != cudaSuccess) {
         g_last_cuda_error = int(e);
         (void)cudaGetLastError();
         return EQUARX_ERR_CUDA;
     }
-    return equarx_allreduce_sim_range(in_bf16, out_bf16, nranks, count, block, g_static_ptr[dev],
+    // (the range call repeats the table checks, now including overlap with the built-in workspace)
+    return equarx_allreduce_sim_range(in_bf16, out_bf16, nranks, count, block, ws,
                                       size_t(EQUARX_STATIC_WORKSPACE_BYTES), 0, 0, nranks, stream);
 }
 

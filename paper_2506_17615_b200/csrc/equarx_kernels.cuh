@@ -51,6 +51,10 @@ __device__ __forceinline__ void st_stream_256(void* p, const Vec8& r) {
 }
 
 // Hop messages are written by one step and read by the next: ask L2 to keep them.
+// They are read with plain (coherent) loads, never through the read-only path: under
+// programmatic dependent launch the reading grid can already be resident while the grid
+// before it is still writing those bytes, and the message slots are reused every two steps,
+// so the data is not read-only for the lifetime of the reading kernel.  L1 is bypassed.
 __device__ __forceinline__ uint64_t policy_keep() {
     uint64_t pol;
     asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
@@ -59,9 +63,10 @@ __device__ __forceinline__ uint64_t policy_keep() {
 
 __device__ __forceinline__ uint4 ld_wire_128(const void* p, uint64_t pol) {
     uint4 r;
-    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.b32 {%0,%1,%2,%3}, [%4], %5;"
+    asm volatile("ld.global.L1::no_allocate.L2::cache_hint.v4.b32 {%0,%1,%2,%3}, [%4], %5;"
                  : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
-                 : "l"(p), "l"(pol));
+                 : "l"(p), "l"(pol)
+                 : "memory");
     return r;
 }
 
@@ -73,7 +78,7 @@ __device__ __forceinline__ void st_wire_128(void* p, const uint4& r, uint64_t po
 
 __device__ __forceinline__ float ld_scale(const float* p, uint64_t pol) {
     float r;
-    asm volatile("ld.global.nc.L2::cache_hint.f32 %0, [%1], %2;" : "=f"(r) : "l"(p), "l"(pol));
+    asm volatile("ld.global.L1::no_allocate.L2::cache_hint.f32 %0, [%1], %2;" : "=f"(r) : "l"(p), "l"(pol) : "memory");
     return r;
 }
 
@@ -243,7 +248,7 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 // lanes 127/amax; the operands are selected, the instruction stream is the same) and
 // the pair of lanes exchanges the quotients with two shuffles.
 template <int LPB>
-__device__ __forceinline__ void quantize_lane(const float (&v)[16], uint4& codes, float& scale, float neg_zero) {
+__device__ __forceinline__ void block_scale_and_inverse(const float (&v)[16], float& scale, float& inv) {
     float m = max3(fabsf(v[0]), fabsf(v[1]), fabsf(v[2]));
     float m1 = max3(fabsf(v[3]), fabsf(v[4]), fabsf(v[5]));
     float m2 = max3(fabsf(v[6]), fabsf(v[7]), fabsf(v[8]));
@@ -253,10 +258,20 @@ __device__ __forceinline__ void quantize_lane(const float (&v)[16], uint4& codes
     m = max3(m, m1, fmaxf(m2, m3));
     m = block_max<LPB>(m);
     const bool odd = threadIdx.x & 1u;
-    const float quot = __fdiv_rn(odd ? 127.0f : m, odd ? m : 127.0f);
-    const float keep = m >= 0x1p-118f ? quot : 0.0f;      // flush rule: scale = inv = 0
+    // a flushed block (amax below 2^-118, zero included) divides 1.0 instead: its quotient is
+    // discarded, and the division never leaves its fast path on zeros and subnormals
+    const bool live = m >= 0x1p-118f;
+    const float ms = live ? m : 1.0f;
+    const float quot = __fdiv_rn(odd ? 127.0f : ms, odd ? ms : 127.0f);
+    const float keep = live ? quot : 0.0f;                // flush rule: scale = inv = 0
     scale = __shfl_sync(0xFFFFFFFFu, keep, (threadIdx.x & 30u));
-    const float inv = __shfl_sync(0xFFFFFFFFu, keep, (threadIdx.x & 30u) | 1u);
+    inv = __shfl_sync(0xFFFFFFFFu, keep, (threadIdx.x & 30u) | 1u);
+}
+
+template <int LPB>
+__device__ __forceinline__ void quantize_lane(const float (&v)[16], uint4& codes, float& scale, float neg_zero) {
+    float inv;
+    block_scale_and_inverse<LPB>(v, scale, inv);
     uint32_t b[16];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -280,6 +295,23 @@ __device__ __forceinline__ void quantize_lane(const float (&v)[16], uint4& codes
         o[j] = __byte_perm(lo, hi, 0x5410);
     }
     codes = make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+// The same quantization with every code kept as the fp32 value of the int8 code (an integer in
+// [-127, 127]) instead of a packed byte: r = fl(fl(v * inv) + 1.5 * 2^23) holds the code in its
+// low mantissa bits, and r - 1.5 * 2^23 is exact and equals (float)code, +0.0 for code 0.  Used
+// where the message is consumed by the lane that produced it and never leaves the registers.
+template <int LPB>
+__device__ __forceinline__ void quantize_lane_values(const float (&v)[16], float (&q)[16], float& scale, float neg_zero) {
+    float inv;
+    block_scale_and_inverse<LPB>(v, scale, inv);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        float t0, t1, r0, r1;
+        fma2_rn(t0, t1, v[2 * i], v[2 * i + 1], inv, neg_zero, neg_zero);      // see quantize_lane
+        add2_rn(r0, r1, t0, t1, 12582912.0f);
+        add2_rn(q[2 * i], q[2 * i + 1], r0, r1, -12582912.0f);
+    }
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
@@ -351,8 +383,10 @@ __device__ __forceinline__ void quantize_lane_payload(const float (&v)[16], uint
     m = max3(m, m1, fmaxf(m2, m3));
     m = block_max<LPB>(m);
     const bool odd = threadIdx.x & 1u;
-    const float quot = __fdiv_rn(odd ? Fp8Format<F>::kMax : m, odd ? m : Fp8Format<F>::kMax);
-    const float keep = m >= Fp8Format<F>::kFlush ? quot : 0.0f;
+    const bool live = m >= Fp8Format<F>::kFlush;
+    const float ms = live ? m : 1.0f;
+    const float quot = __fdiv_rn(odd ? Fp8Format<F>::kMax : ms, odd ? ms : Fp8Format<F>::kMax);
+    const float keep = live ? quot : 0.0f;
     scale = __shfl_sync(0xFFFFFFFFu, keep, (threadIdx.x & 30u));
     const float inv = __shfl_sync(0xFFFFFFFFu, keep, (threadIdx.x & 30u) | 1u);
     uint32_t o[4];
@@ -392,8 +426,8 @@ __device__ __forceinline__ Vec8 dequant_to_bf16_payload(const uint4& c, float sc
 // SPLIT   (the per-step entry points): codes[count] and scales[count/B] are separate arrays.
 // RECORDS (the simulations): a message is a sequence of 544-byte records, one per tile of
 //         512 elements: 8 floats of metadata first (the tile's 512/B scales, zero padded to
-//         one 32-byte sector), then the 512 codes ("send the metadata before any
-//         microshards", Section 3.1).  Every sector of a record is written whole, so a
+//         one 32-byte sector), then the 512 codes (Section 3.1 sends metadata ahead of
+//         the microshards it describes).  Every sector of a record is written whole, so a
 //         message that is read back while it is still in L2 never needs a fill from DRAM.
 constexpr int kTileElems = 512;
 constexpr int kRecordHeader = 32;
@@ -437,11 +471,10 @@ struct GatherArgs {
 struct PipeArgs {
     const void* in[kMaxRanks];       // input tensor of rank r (whole tensor)
     void* out[kMaxRanks];            // output tensor of rank r
-    char* records;                   // trace: record region [shard k][event j][tile]; else per-warp FIFOs
+    char* records;                   // the trace: record region [shard k][event j][tile] (unused by the chain-fused form)
     uint64_t shard;
     uint64_t tiles_per_shard;        // 512-element tiles per shard (the last one may be ragged)
     uint32_t nranks;
-    uint32_t keep_trace;
     float neg_zero;                  // -0.0f, opaque to the compiler (see quantize_lane)
 };
 
@@ -536,23 +569,20 @@ __global__ void __launch_bounds__(kThreads) ag_dequant_kernel(const __grid_const
     for (uint32_t r = 0; r < a.nranks; ++r) st_stream_256(static_cast<char*>(a.out[r]) + byte_off, o);
 }
 
-// Deep-pipelined form of the whole schedule (Section 3.1 pipelines the microshards of a
-// shard through the ring independently; here a microshard is one tile of 512 elements).
-// One warp carries its tile through all N ring steps and the all-gather without waiting
-// for any other tile.  Every hop message still goes through memory as a record: the lane
-// that acts for the sending rank stores its codes (and lanes 0..7 the metadata sector),
-// the warp synchronises, and the NEIGHBOURING lane (lane ^ 1), acting for the receiving
-// rank, loads them back and continues with that 16-element group.  Without a trace the
-// records go to a two-deep staging FIFO that the warp owns and reuses for every step
-// and every tile, the way a ring channel reuses its staging buffers: the FIFO stays in
-// L2 and the hop traffic never reaches HBM.  With a trace every message is kept.
-// The bf16 shard of the next step is prefetched while a step computes.
+// Deep-pipelined form of the whole schedule with every message kept (Section 3.1 pipelines the
+// microshards of a shard through the ring independently; here a microshard is one tile of 512
+// elements).  One warp carries its tile through all N ring steps and the all-gather without
+// waiting for any other tile.  Every hop message goes through memory as a record of the trace:
+// the lane that acts for the sending rank stores its codes (and lanes 0..7 the metadata sector),
+// the warp synchronises, and the NEIGHBOURING lane (lane ^ 1), acting for the receiving rank,
+// loads them back and continues with that 16-element group.  The bf16 shard of the next step is
+// prefetched while a step computes.
 constexpr int kPipeThreads = 64;
 #ifndef EQX_PIPE_MINBLOCKS
 #define EQX_PIPE_MINBLOCKS 18
 #endif
 
-template <int LPB, bool TRACE>
+template <int LPB>
 __global__ void __launch_bounds__(kPipeThreads, EQX_PIPE_MINBLOCKS) pipelined_kernel(const __grid_constant__ PipeArgs a) {
     const uint32_t lane = threadIdx.x & 31u;
     const uint64_t warps = (uint64_t)gridDim.x * (kPipeThreads / 32);
@@ -561,7 +591,6 @@ __global__ void __launch_bounds__(kPipeThreads, EQX_PIPE_MINBLOCKS) pipelined_ke
     const uint64_t groups = a.shard >> 4;
     const uint64_t tiles = a.tiles_per_shard * N;
     const uint64_t trace_stride = a.tiles_per_shard * kRecordBytes;      // one event further in the trace
-    char* const fifo = a.records + warp * (2 * kRecordBytes);
     // byte offsets inside a record: even steps send from position `lane` and receive (as the
     // neighbouring lane, acting for the receiving rank) at position lane ^ 1; odd steps the reverse
     const uint32_t code_own = kRecordHeader + lane * 16, code_nbr = kRecordHeader + (lane ^ 1u) * 16;
@@ -594,8 +623,7 @@ __global__ void __launch_bounds__(kPipeThreads, EQX_PIPE_MINBLOCKS) pipelined_ke
         const uint64_t off_own = off_next;
         const bool active = off_own != ~uint64_t(0);   // lane pairs are in or out together (groups % 4 == 0)
         const uint64_t off_nbr = off_own ^ 32;         // the neighbouring lane's group
-        char* trace = TRACE ? a.records + ((uint64_t)k * N * a.tiles_per_shard + (tile - (uint64_t)k * a.tiles_per_shard)) * kRecordBytes
-                            : nullptr;
+        char* trace = a.records + ((uint64_t)k * N * a.tiles_per_shard + (tile - (uint64_t)k * a.tiles_per_shard)) * kRecordBytes;
         uint32_t rho = k + 1 == N ? 0 : k + 1;         // rank of step 0
         float v[16];
         widen_bf16x16(xw, v);
@@ -629,8 +657,6 @@ __global__ void __launch_bounds__(kPipeThreads, EQX_PIPE_MINBLOCKS) pipelined_ke
                 c = ld_coherent_128(rec + code_recv);
                 s = ld_coherent_f32(reinterpret_cast<const float*>(rec + scale_recv));
             }
-            // a FIFO entry is overwritten two steps later, after the __syncwarp of the step in between:
-            // every lane's load above has returned by then, because its value feeds that step's quantization
         };
         auto gather = [&](const uint4& c, float s, uint64_t off) {      // all-gather: one store per rank
             const Vec8 o = dequant_to_bf16x16(c, s);
@@ -643,26 +669,133 @@ __global__ void __launch_bounds__(kPipeThreads, EQX_PIPE_MINBLOCKS) pipelined_ke
             float s;
             // even step: send from the own position, receive at the neighbour's
             prefetch(j, off_nbr);
-            exchange(TRACE ? trace : fifo, hdr_src_even, code_own, code_nbr, scale_nbr, c, s);
+            exchange(trace, hdr_src_even, code_own, code_nbr, scale_nbr, c, s);
             if (j + 1 == N) {
                 gather(c, s, off_nbr);
                 break;
             }
             widen_bf16x16(xw, v);
             dequant_add_x16(c, s, v);
-            if (TRACE) trace += trace_stride;
+            trace += trace_stride;
             // odd step: send from the neighbour's position, receive at the own
             prefetch(j + 1, off_own);
-            exchange(TRACE ? trace : fifo + kRecordBytes, hdr_src_odd, code_nbr, code_own, scale_own, c, s);
+            exchange(trace, hdr_src_odd, code_nbr, code_own, scale_own, c, s);
             if (j + 2 == N) {
                 gather(c, s, off_own);
                 break;
             }
             widen_bf16x16(xw, v);
             dequant_add_x16(c, s, v);
-            if (TRACE) trace += trace_stride;
+            trace += trace_stride;
         }
-        __syncwarp();                                  // the next tile reuses the FIFO
+    }
+}
+
+// Chain-fused form of the same schedule, used when no trace is kept.  A tile's adder chain
+// (Section 3.3, Fig. 4) depends on no other tile, so the lane that quantized a 16-element group
+// for the sending rank can go on, as the receiving rank, with the fused multiply-add on that
+// rank's counterpart: the hop message of a group (its codes, as the fp32 values of the int8
+// codes, and the block's scale) stays in that lane's registers and is never stored.  Codes,
+// scales and outputs are bit for bit those of pipelined_kernel<LPB, true>, which writes every
+// message as a record and is the witness of that; what this kernel moves through HBM is the
+// bf16 inputs once and the bf16 outputs once (4 bytes per element of every rank).
+// The bf16 shard of the next rank of the chain is in flight while a step computes; DEPTH is the
+// number of such loads in flight per lane.
+#ifndef EQX_FUSED_MINBLOCKS
+#define EQX_FUSED_MINBLOCKS 18
+#endif
+#ifndef EQX_FUSED_DEPTH
+#define EQX_FUSED_DEPTH 1
+#endif
+
+// QUANT = false is the unquantized comparator in the same form: the message is the partial sum
+// rounded to bf16 and the receiving rank's add is rounded to bf16 again (the BF16 baseline's hop).
+template <int LPB, int DEPTH, bool QUANT>
+__global__ void __launch_bounds__(kPipeThreads, EQX_FUSED_MINBLOCKS) chain_fused_kernel(const __grid_constant__ PipeArgs a) {
+    static_assert(DEPTH == 1 || DEPTH == 2, "one or two shards in flight");
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint64_t warps = (uint64_t)gridDim.x * (kPipeThreads / 32);
+    const uint64_t warp = (uint64_t)blockIdx.x * (kPipeThreads / 32) + (threadIdx.x >> 5);
+    const uint32_t N = a.nranks;
+    const uint64_t groups = a.shard >> 4;
+    const uint64_t tiles = a.tiles_per_shard * N;
+
+    pdl_launch_dependents();
+    pdl_wait_prior_grid();           // nothing is read before the previous kernel of the stream has completed
+
+    // byte offset of this lane's group of a tile in every rank's tensor; ~0 past the end of a ragged last tile
+    auto offset_of = [&](uint64_t tile_, uint32_t& k_) -> uint64_t {
+        k_ = (uint32_t)(tile_ / a.tiles_per_shard);
+        const uint64_t t_ = tile_ - (uint64_t)k_ * a.tiles_per_shard;
+        if (t_ * 32 + lane >= groups) return ~uint64_t(0);
+        return ((uint64_t)k_ * a.shard + (t_ * 32 + lane) * 16) * 2;
+    };
+    auto load = [&](uint32_t rank, uint64_t off) {
+        Vec8 x = {};
+        if (off != ~uint64_t(0)) x = ld_coherent_256(static_cast<const char*>(a.in[rank]) + off);   // in place is allowed: no read-only path
+        return x;
+    };
+    auto next_rank = [&](uint32_t r) { return r + 1 == N ? 0u : r + 1; };
+
+    // The loads of a tile run over the chain's ranks k+1, k+2, ..., k; when they are used up, the
+    // stream of loads continues with the warp's next tile, so DEPTH loads are always in flight.
+    uint64_t tile_ld = warp;                    // tile, rank and offset of the next load to issue
+    uint32_t k_ld = 0, left_ld = N;             // left_ld: loads of tile_ld still to issue
+    uint64_t off_ld = tile_ld < tiles ? offset_of(tile_ld, k_ld) : ~uint64_t(0);
+    uint32_t rank_ld = next_rank(k_ld);
+    auto issue = [&]() {
+        const Vec8 x = load(rank_ld, tile_ld < tiles ? off_ld : ~uint64_t(0));
+        rank_ld = next_rank(rank_ld);
+        if (--left_ld == 0) {
+            tile_ld += warps;
+            left_ld = N;
+            off_ld = tile_ld < tiles ? offset_of(tile_ld, k_ld) : ~uint64_t(0);
+            rank_ld = next_rank(k_ld);
+        }
+        return x;
+    };
+
+    Vec8 x0 = issue(), x1 = {};
+    if (DEPTH == 2) x1 = issue();
+
+    for (uint64_t tile = warp; tile < tiles; tile += warps) {
+        uint32_t k;
+        const uint64_t off = offset_of(tile, k);
+        float v[16];                            // the partial sum, then (in place) the code values of its message
+        widen_bf16x16(x0, v);                   // rank k+1's shard opens the chain
+        if (DEPTH == 2) { x0 = x1; x1 = issue(); } else { x0 = issue(); }
+        float scale = 0.0f;
+        for (uint32_t j = 1;; ++j) {
+            if (QUANT) quantize_lane_values<LPB>(v, v, scale, a.neg_zero);      // the message of step j-1
+            if (j == N) break;
+            if (QUANT) {
+                // the receiving rank: v = fma(code, scale, its counterpart), straight from the bf16 words
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    fma2_rn(v[2 * i], v[2 * i + 1], v[2 * i], v[2 * i + 1], scale,
+                            __uint_as_float(x0.w[i] << 16), __uint_as_float(x0.w[i] & 0xFFFF0000u));
+            } else {
+                // v holds bf16 values (a raw shard, or a rounded sum): the message is v itself
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const uint32_t sum = pack_bf16x2_rn(__fadd_rn(v[2 * i], __uint_as_float(x0.w[i] << 16)),
+                                                        __fadd_rn(v[2 * i + 1], __uint_as_float(x0.w[i] & 0xFFFF0000u)));
+                    v[2 * i] = __uint_as_float(sum << 16);
+                    v[2 * i + 1] = __uint_as_float(sum & 0xFFFF0000u);
+                }
+            }
+            if (DEPTH == 2) { x0 = x1; x1 = issue(); } else { x0 = issue(); }
+        }
+        // all-gather: the last message, dequantized (or forwarded as it is), goes to every rank
+        Vec8 o;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float lo = v[2 * i], hi = v[2 * i + 1];
+            if (QUANT) mul2_rn(lo, hi, v[2 * i], v[2 * i + 1], scale);
+            o.w[i] = pack_bf16x2_rn(lo, hi);
+        }
+        if (off != ~uint64_t(0))
+            for (uint32_t r = 0; r < N; ++r) st_stream_256(static_cast<char*>(a.out[r]) + off, o);
     }
 }
 
@@ -856,6 +989,118 @@ __global__ void __launch_bounds__(kPipeThreads) flavour_kernel(const __grid_cons
             for (uint32_t r = 0; r < N; ++r) st_stream_256(static_cast<char*>(a.out[r]) + byte_off, o);
         }
         __syncwarp();                      // the next tile reuses the FIFO
+    }
+}
+
+// The same flavours with every message kept in registers (used when no trace is asked for): the
+// lane that produced a group's message goes on as the receiving rank, as in chain_fused_kernel.
+// One hop: the message of v (quantized with the flavour's payload, or rounded to bf16) is folded
+// into `addend` by the receiver; `out` may be v or addend.
+template <int LPB, int PAYLOAD>
+__device__ __forceinline__ void fused_hop(const float (&v)[16], const float (&addend)[16], float (&out)[16],
+                                          float neg_zero) {
+    if (PAYLOAD == 1) {
+        float q[16], scale;
+        quantize_lane_values<LPB>(v, q, scale, neg_zero);
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            fma2_rn(out[2 * i], out[2 * i + 1], q[2 * i], q[2 * i + 1], scale, addend[2 * i], addend[2 * i + 1]);
+    } else if (PAYLOAD != 0) {
+        uint4 codes;
+        float q[16], scale;
+        quantize_lane_payload<LPB, PAYLOAD == 0 ? 2 : PAYLOAD>(v, codes, scale, neg_zero);
+        decode_x16<PAYLOAD == 0 ? 2 : PAYLOAD>(codes, q);
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            fma2_rn(out[2 * i], out[2 * i + 1], q[2 * i], q[2 * i + 1], scale, addend[2 * i], addend[2 * i + 1]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t m = pack_bf16x2_rn(v[2 * i], v[2 * i + 1]);                  // the bf16 message
+            const uint32_t sum = pack_bf16x2_rn(__fadd_rn(__uint_as_float(m << 16), addend[2 * i]),
+                                                __fadd_rn(__uint_as_float(m & 0xFFFF0000u), addend[2 * i + 1]));
+            out[2 * i] = __uint_as_float(sum << 16);
+            out[2 * i + 1] = __uint_as_float(sum & 0xFFFF0000u);
+        }
+    }
+}
+
+template <int LPB, bool SEMI, bool QRS, bool QAG, int PAYLOAD>
+__global__ void __launch_bounds__(kPipeThreads) flavour_fused_kernel(const __grid_constant__ FlavourArgs a) {
+    constexpr int RS = QRS ? PAYLOAD : 0;
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint64_t warps = (uint64_t)gridDim.x * (kPipeThreads / 32);
+    const uint64_t warp = (uint64_t)blockIdx.x * (kPipeThreads / 32) + (threadIdx.x >> 5);
+    const uint32_t N = a.nranks;
+    const uint32_t h = N / 2;
+    const uint64_t groups = a.shard >> 4;
+    const uint64_t tiles = a.tiles_per_shard * N;
+
+    for (uint64_t tile = warp; tile < tiles; tile += warps) {
+        const uint32_t k = (uint32_t)(tile / a.tiles_per_shard);
+        const uint64_t t = tile - (uint64_t)k * a.tiles_per_shard;
+        const bool active = t * 32 + lane < groups;
+        const uint64_t off = ((uint64_t)k * a.shard + (t * 32 + lane) * 16) * 2;    // this lane's group, in bytes
+        auto fetch = [&](uint32_t rank) {
+            Vec8 x = {};
+            if (active) x = ld_coherent_256(static_cast<const char*>(a.in[rank % N]) + off);
+            return x;
+        };
+        // a chain: v starts as rank `first`'s shard and hops through `hops` further ranks (rank first + dir * j)
+        auto run_chain = [&](float (&v)[16], uint32_t first, int dir, uint32_t hops) {
+            {
+                const Vec8 x0 = fetch(first);
+                widen_bf16x16(x0, v);
+            }
+            if (hops == 0) return;
+            Vec8 nx = fetch(first + N + dir);
+            for (uint32_t j = 1; j <= hops; ++j) {
+                float x[16];
+                widen_bf16x16(nx, x);
+                if (j < hops) nx = fetch(first + N * (j + 1) + dir * (int)(j + 1));   // next counterpart, in flight
+                fused_hop<LPB, RS>(v, x, v, a.neg_zero);
+            }
+        };
+
+        float acc[16];                     // the owner's reduced group
+        if (!SEMI) {
+            run_chain(acc, k + 1, +1, N - 1);                       // k+1 -> k+2 -> ... -> k
+        } else {
+            {
+                const Vec8 xo = fetch(k);
+                widen_bf16x16(xo, acc);
+            }
+            float v[16];
+            if (h >= 2) {                                           // chain B: k+h+1 -> ... -> k+N-1 -> owner
+                run_chain(v, k + h + 1, +1, h - 2);
+                fused_hop<LPB, RS>(v, acc, acc, a.neg_zero);
+            }
+            run_chain(v, k + h, -1, h - 1);                         // chain A: k+h -> ... -> k+1 -> owner
+            fused_hop<LPB, RS>(v, acc, acc, a.neg_zero);
+        }
+
+        // all-gather: one more quantize/dequantize pair, or the sum rounded to bf16
+        Vec8 o;
+        if (QAG && PAYLOAD == 1) {
+            float q[16], scale;
+            quantize_lane_values<LPB>(acc, q, scale, a.neg_zero);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                float lo, hi;
+                mul2_rn(lo, hi, q[2 * i], q[2 * i + 1], scale);
+                o.w[i] = pack_bf16x2_rn(lo, hi);
+            }
+        } else if (QAG) {
+            uint4 codes;
+            float scale;
+            quantize_lane_payload<LPB, PAYLOAD>(acc, codes, scale, a.neg_zero);
+            o = dequant_to_bf16_payload<PAYLOAD>(codes, scale);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) o.w[i] = pack_bf16x2_rn(acc[2 * i], acc[2 * i + 1]);
+        }
+        if (active)
+            for (uint32_t r = 0; r < N; ++r) st_stream_256(static_cast<char*>(a.out[r]) + off, o);
     }
 }
 

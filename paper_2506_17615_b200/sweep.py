@@ -4,10 +4,12 @@
 
 For every point (N in {4, 8, 16}, block in {128, 256, 512}, uniform(-1,1) and N(0,1), per-rank
 messages from 16 KB to 256 MB in powers of two) it times, with CUDA events and inputs resident in
-device memory, the pipelined schedule, the launch-per-step schedule and the unquantized bf16 ring,
-and prints one JSON line per point: GB/s of bf16 input reduced and the fraction of the HBM
-roofline (algorithmic bytes n*N*(6+8/B) over the measured copy bandwidth).  Inputs rotate over
-several resident sets so that consecutive iterations do not find their inputs in L2.
+device memory, the single-launch (chain-fused) schedule, the launch-per-step schedule and the
+unquantized bf16 ring, and prints one JSON line per point: GB/s of bf16 input reduced and the
+fraction of the HBM roofline, each schedule against the bytes it must move: 4*n*N for the single
+launch (inputs once, outputs once; its hop messages stay in registers), n*N*(6+8/B) for the
+launch-per-step schedule, n*(8N-4) for the bf16 ring, over the measured copy bandwidth.  Inputs
+rotate over several resident sets so that consecutive iterations do not find their inputs in L2.
 """
 import argparse
 import json
@@ -71,10 +73,11 @@ def run_point(n_ranks, nbytes, block, dist, peak):
     t_bf16 = time_ms(lambda i: eq.allreduce_sim_bf16(ins[i % sets], outs[i % sets], n_ranks, count,
                                                      ws16, wb16, stream), iters)
     alg = count * n_ranks * (6 + 8 / block)
+    fused = 4 * count * n_ranks
     alg16 = count * (8 * n_ranks - 4)
     gbs = lambda nbytes_, ms: nbytes_ / (ms * 1e-3) / 1e9
     return {"nranks": n_ranks, "bytes_per_rank": nbytes, "block": block, "dist": dist, "iters": iters, "sets": sets,
-            "pipelined": {"ms": t_pipe, "gbs_in": gbs(in_bytes, t_pipe), "frac": gbs(alg, t_pipe) / peak},
+            "pipelined": {"ms": t_pipe, "gbs_in": gbs(in_bytes, t_pipe), "frac": gbs(fused, t_pipe) / peak},
             "by_steps": {"ms": t_steps, "gbs_in": gbs(in_bytes, t_steps), "frac": gbs(alg, t_steps) / peak},
             "bf16_sim": {"ms": t_bf16, "gbs_in": gbs(in_bytes, t_bf16), "frac": gbs(alg16, t_bf16) / peak}}
 
@@ -86,11 +89,12 @@ def summarize(path):
     out = ["# Message-size sweep (config 4): GB/s of bf16 input reduced and fraction of the HBM roofline",
            "",
            "Command: `python -m paper_2506_17615_b200.sweep --out sweep.jsonl` on one B200 (CUDA events, inputs resident,",
-           "several input/output sets in rotation), then `--summarize sweep.jsonl`. Fraction = algorithmic bytes n*N*(6+8/B)",
-           f"(bf16 comparator: n*(8N-4)) over time, divided by the {rows[0]['peak_source']} HBM copy bandwidth {peak:.1f} GB/s.",
+           "several input/output sets in rotation), then `--summarize sweep.jsonl`. Fraction = bytes the schedule must move",
+           "(single launch, chain-fused: 4*n*N; launch per step: n*N*(6+8/B); bf16 comparator: n*(8N-4)) over time,",
+           f"divided by the {rows[0]['peak_source']} HBM copy bandwidth {peak:.1f} GB/s.",
            f"{len(rows)} points; the table lists N(0,1) data (uniform(-1,1) is within a few percent).",
            "",
-           "| N | block | bytes per rank | pipelined GB/s (frac) | launch per step GB/s (frac) | bf16 ring per step GB/s (frac) |",
+           "| N | block | bytes per rank | single launch GB/s (frac) | launch per step GB/s (frac) | bf16 ring per step GB/s (frac) |",
            "|---|---|---|---|---|---|"]
     shown = (1 << 14, 1 << 17, 1 << 20, 1 << 22, 1 << 24, 1 << 26, 1 << 27, 1 << 28)
     for r in rows:
@@ -105,11 +109,11 @@ def summarize(path):
         lo = lambda key: min(r[key]["frac"] for r in big)
         hi = lambda key: max(r[key]["frac"] for r in big)
         out += ["",
-                f"All {len(big)} points with at least 64 MB per rank: pipelined {lo('pipelined'):.3f} - {hi('pipelined'):.3f} of the "
+                f"All {len(big)} points with at least 64 MB per rank: single launch {lo('pipelined'):.3f} - {hi('pipelined'):.3f} of the "
                 f"measured peak ({lo('pipelined') * peak / 8000:.3f} - {hi('pipelined') * peak / 8000:.3f} of the nominal 8 TB/s); "
                 f"launch per step {lo('by_steps'):.3f} - {hi('by_steps'):.3f} of measured "
                 f"({lo('by_steps') * peak / 8000:.3f} - {hi('by_steps') * peak / 8000:.3f} of nominal). Below about 2 MB per rank "
-                "every schedule is launch- and latency-bound (the paper sees the same below 2 MiB, Section 4); the pipelined "
+                "every schedule is launch- and latency-bound (the paper sees the same below 2 MiB, Section 4); the single-launch "
                 "schedule needs one launch instead of N+1 there."]
     return "\n".join(out) + "\n"
 

@@ -89,6 +89,27 @@ int main(void)
             return 1;
         }
     }
+    /* host buffers in, host buffers out: pageable memory here, so the copies are synchronous */
+    {
+        void *stage;
+        const size_t sb = equarx_allreduce_sim_host_staging_bytes(N, count);
+        if (sb != 2 * count * N) return 1;
+        CHECK_CUDA(cudaMalloc(&stage, sb));
+        CHECK_EQ(equarx_oracle_allreduce((const uint16_t *const *)h_in, h_ref, N, count, BLOCK, NULL, NULL, NULL));
+        for (int r = 0; r < N; ++r) memset(h_out[r], 0xEE, count * 2);
+        CHECK_EQ(equarx_allreduce_sim_host((const void *const *)h_in, (void *const *)h_out, N, count, BLOCK, stage, sb,
+                                           NULL));
+        CHECK_CUDA(cudaDeviceSynchronize());
+        for (int r = 0; r < N; ++r)
+            if (memcmp(h_out[r], h_ref[r], count * 2) != 0) {
+                fprintf(stderr, "host-buffer AllReduce output of rank %d differs\n", r);
+                return 1;
+            }
+        if (equarx_allreduce_sim_host((const void *const *)h_in, (void *const *)h_out, N, count, BLOCK, stage, sb - 1,
+                                      NULL) != EQUARX_ERR_WORKSPACE)
+            return 1;
+        CHECK_CUDA(cudaFree(stage));
+    }
     /* an error path: a count that is not a multiple of nranks * block is refused before any launch */
     if (equarx_allreduce_sim((const void *const *)d_in, d_out, N, count + BLOCK, BLOCK, d_out[0], 1 << 20, 0, NULL)
         != EQUARX_ERR_COUNT)

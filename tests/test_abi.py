@@ -50,7 +50,7 @@ def test_workspace_bytes():
     assert eq.allreduce_sim_workspace_bytes(3, 65536, 256, False) == 0      # not divisible
     assert eq.allreduce_sim_workspace_bytes(4, 65536, 100, False) == 0
     assert eq.allreduce_sim_workspace_bytes(65, 65 * 256, 256, False) == 0
-    assert eq.allreduce_sim_pipelined_workspace_bytes(4, 65536, 256, False) == binding.PIPELINE_FIFO_BYTES
+    assert eq.allreduce_sim_pipelined_workspace_bytes(4, 65536, 256, False) == binding.PIPELINE_MIN_WORKSPACE_BYTES
     assert eq.allreduce_sim_pipelined_workspace_bytes(4, 65536, 256, True) == 16 * 32 * 544
     assert eq.allreduce_sim_pipelined_workspace_bytes(4, 65536, 99, True) == 0
     assert eq.allreduce_sim_bf16_workspace_bytes(4, 65536) == 4 * 65536
@@ -155,6 +155,46 @@ def test_bf16_sim_rejects_bad_arguments():
     assert status_of(f, ins, outs, 4, 65536, 0, 4 * 65536) == binding.ERR_NULL
     assert status_of(f, ins, outs, 4, 65536, ws, 4 * 65536 - 1) == binding.ERR_WORKSPACE
     assert status_of(f, ins, [ins[1]] + outs[1:], 4, 65536, ws, 4 * 65536) == binding.ERR_ALIAS
+
+
+def test_host_entry_rejects_bad_arguments():
+    """equarx_allreduce_sim_host validates before any copy is enqueued."""
+    f = eq.allreduce_sim_host
+    H = 0x5000_0000_0000           # made-up host addresses
+    hin = [H + r * MB for r in range(4)]
+    hout = [H + (16 + r) * MB for r in range(4)]
+    stage = A
+    sb = eq.allreduce_sim_host_staging_bytes(4, 65536)
+    assert sb == 2 * 65536 * 4
+    assert eq.allreduce_sim_host_staging_bytes(0, 65536) == 0
+    assert status_of(f, hin, hout, 0, 65536, 256, stage, sb) == binding.ERR_NRANKS
+    assert status_of(f, hin, hout, 4, 65536, 96, stage, sb) == binding.ERR_BLOCK
+    assert status_of(f, hin, hout, 4, 65536 + 256, 256, stage, sb + 4096) == binding.ERR_COUNT
+    assert status_of(f, hin, hout, 4, 65536, 256, 0, sb) == binding.ERR_NULL
+    assert status_of(f, hin[:3] + [0], hout, 4, 65536, 256, stage, sb) == binding.ERR_NULL
+    assert status_of(f, None, hout, 4, 65536, 256, stage, sb) == binding.ERR_NULL
+    assert status_of(f, hin, hout, 4, 65536, 256, stage, sb - 1) == binding.ERR_WORKSPACE
+    assert status_of(f, hin, hout, 4, 65536, 256, stage + 16, sb) == binding.ERR_ALIGN
+    assert status_of(f, [hin[0] + 1] + hin[1:], hout, 4, 65536, 256, stage, sb) == binding.ERR_ALIGN
+    assert status_of(f, hin, [hin[1]] + hout[1:], 4, 65536, 256, stage, sb) == binding.ERR_ALIAS
+    assert status_of(f, hin, [hout[1]] + hout[1:], 4, 65536, 256, stage, sb) == binding.ERR_ALIAS
+
+
+def test_static_entry_validates_before_any_cuda_call():
+    """NULL, misaligned and aliased tables, and problems beyond the built-in workspace, are
+    rejected on the host: these calls run on a machine without a GPU."""
+    f = eq.allreduce_sim_static
+    a = sim_args()
+    ins, outs = a["in_bf16"], a["out_bf16"]
+    assert status_of(f, ins[:3] + [0], outs, 4, 65536, 256) == binding.ERR_NULL
+    assert status_of(f, None, outs, 4, 65536, 256) == binding.ERR_NULL
+    assert status_of(f, ins, [outs[0] + 16] + outs[1:], 4, 65536, 256) == binding.ERR_ALIGN
+    assert status_of(f, ins, [ins[1]] + outs[1:], 4, 65536, 256) == binding.ERR_ALIAS
+    assert status_of(f, ins, outs, 4, 65536, 100) == binding.ERR_BLOCK
+    big = 8 * 256 * 4096 * 4            # needs more than 16 MiB of message slots
+    assert eq.allreduce_sim_workspace_bytes(8, big, 256) > binding.STATIC_WORKSPACE_BYTES
+    assert status_of(f, [A] * 8, [A] * 8, 8, big, 256) == binding.ERR_STATIC_LIMIT
+    assert eq.last_cuda_error() == 0
 
 
 def test_no_cuda_error_recorded_by_validation():

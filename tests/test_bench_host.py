@@ -18,12 +18,13 @@ import bench  # noqa: E402
 def test_algorithmic_bytes_match_the_closed_form():
     # n * N * (6 + 8/B); config 3: N=8, n=8192*5376, B=256 -> 2124.9 MB
     n, N, B = 8192 * 5376, 8, 256
-    assert bench.algorithmic_bytes(N, n, B) == n * N * (6 + 8 / B)
-    assert round(bench.algorithmic_bytes(N, n, B) / 1e6, 1) == 2124.9
+    assert bench.ring_schedule_bytes(N, n, B) == n * N * (6 + 8 / B)
+    assert round(bench.ring_schedule_bytes(N, n, B) / 1e6, 1) == 2124.9
+    assert bench.chain_fused_bytes(N, n) == 4 * n * N
     total = (bench.launch_bytes("quantize_blocks", N, n, B)
              + (N - 1) * bench.launch_bytes("rs_step_dequant_add_requant", N, n, B)
              + bench.launch_bytes("ag_dequant", N, n, B))
-    assert total == bench.algorithmic_bytes(N, n, B)
+    assert total == bench.ring_schedule_bytes(N, n, B)
 
 
 def test_aggregate_value_is_whole_job():
@@ -74,7 +75,7 @@ def test_sweep_summary_from_a_results_file(tmp_path):
     """The sweep's markdown summary is plain host code: feed it two fabricated result lines."""
     from paper_2506_17615_b200 import sweep
     rows = []
-    for nbytes, frac in ((1 << 20, 0.4), (1 << 26, 1.3)):
+    for nbytes, frac in ((1 << 20, 0.4), (1 << 26, 0.96)):
         leg = {"ms": 1.0, "gbs_in": 1000.0, "frac": frac}
         rows.append({"nranks": 8, "bytes_per_rank": nbytes, "block": 256, "dist": "normal", "iters": 5, "sets": 2,
                      "pipelined": leg, "by_steps": dict(leg, frac=frac * 0.75), "bf16_sim": leg,
@@ -82,5 +83,5 @@ def test_sweep_summary_from_a_results_file(tmp_path):
     path = tmp_path / "sweep.jsonl"
     path.write_text("\n".join(json.dumps(r) for r in rows) + "\n")
     text = sweep.summarize(str(path))
-    assert "| 8 | 256 | 1 MB | 1000 (0.400)" in text and "| 8 | 256 | 64 MB | 1000 (1.300)" in text
-    assert "All 1 points with at least 64 MB per rank: pipelined 1.300 - 1.300" in text
+    assert "| 8 | 256 | 1 MB | 1000 (0.400)" in text and "| 8 | 256 | 64 MB | 1000 (0.960)" in text
+    assert "All 1 points with at least 64 MB per rank: single launch 0.960 - 0.960" in text

@@ -93,18 +93,14 @@ def test_both_quantized_is_the_pipelined_schedule_and_none_is_the_bf16_ring(gu):
 
 
 @pytest.mark.parametrize("flavour", (1, 3, 7))
-def test_semi_loop_full_size_sampled(gu, flavour):
-    """Config 2 at full size through the semi-loop flavours: sampled blocks against the oracle."""
+def test_semi_loop_full_size_every_word(gu, flavour):
+    """Config 2 at full size through the semi-loop flavours: every output word against the oracle."""
     w = wl.C2
     semi, qr, qa = decode(flavour)
     x = wl.make_inputs(w, device="cuda")
     out, _ = run_flavour(gu, x, w.block, flavour, False)
-    picks = gu.sample_blocks(w.nranks, w.count // w.nranks // w.block, 16, seed=flavour)
-    sub = gu.gather_blocks(x, picks, w.block)
-    exp = oracle.allreduce_variant(wl.as_u16(sub), w.block, semi, qr, qa)["out"]
-    gu.assert_same_words(gu.gather_blocks(out, picks, w.block), exp, f"flavour {flavour} sampled")
-    for r in range(1, w.nranks):
-        assert torch.equal(out[0].view(torch.int16), out[r].view(torch.int16))
+    exp = oracle.allreduce_variant(wl.as_u16(x), w.block, semi, qr, qa)["out"]
+    gu.assert_same_words(out, exp, f"flavour {flavour}, config 2")
 
 
 def test_flavour_argument_errors(gu):
@@ -119,7 +115,8 @@ def test_flavour_argument_errors(gu):
         eq.allreduce_sim_flavour(*args, eq.FLAVOUR_SEMI_LOOP, ws, ws.numel())      # odd rank count
     assert e.value.status == binding.ERR_NRANKS
     assert eq.allreduce_sim_flavour_workspace_bytes(3, 3 * 64, 64, 1) == 0
-    assert eq.allreduce_sim_flavour_workspace_bytes(4, 4 * 64, 64, 1) == binding.FLAVOUR_FIFO_BYTES
+    assert eq.allreduce_sim_flavour_workspace_bytes(4, 4 * 64, 64, 1) == binding.PIPELINE_MIN_WORKSPACE_BYTES
+    assert eq.allreduce_sim_flavour_workspace_bytes(4, 4 * 64, 64, 1, True) > binding.FLAVOUR_FIFO_BYTES
 
 
 FP8_FLAVOURS = [sched | fmt for fmt in (eq.FLAVOUR_E4M3, eq.FLAVOUR_E5M2) for sched in (2, 3, 4, 5, 6, 7)]
@@ -152,5 +149,5 @@ def test_fp8_stress_blocks(gu, flavour):
 def test_fp8_flavour_bits_are_validated(gu):
     assert eq.allreduce_sim_flavour_workspace_bytes(4, 4 * 64, 64, eq.FLAVOUR_E4M3) == 0            # nothing quantized
     assert eq.allreduce_sim_flavour_workspace_bytes(4, 4 * 64, 64, 6 | eq.FLAVOUR_E4M3 | eq.FLAVOUR_E5M2) == 0
-    assert eq.allreduce_sim_flavour_workspace_bytes(4, 4 * 64, 64, 6 | eq.FLAVOUR_E5M2) == binding.FLAVOUR_FIFO_BYTES
+    assert eq.allreduce_sim_flavour_workspace_bytes(4, 4 * 64, 64, 6 | eq.FLAVOUR_E5M2) == binding.PIPELINE_MIN_WORKSPACE_BYTES
     assert eq.allreduce_sim_flavour_workspace_bytes(4, 4 * 64, 64, 32) == 0

@@ -156,28 +156,63 @@ def test_in_place(gu):
     _compare_full(gu, wl.make_inputs(w), 256, in_place=True)
 
 
+@pytest.fixture(scope="module")
+def full_size_expected():
+    """Oracle outputs of the full-size configs, computed once per test session (the oracle
+    evaluates all of config 2 in well under a second and all of config 3 in a few seconds)."""
+    cache = {}
+
+    def get(w):
+        if w.name not in cache:
+            x = wl.make_inputs(w, device="cuda")
+            cache.clear()                                   # one config's host copy at a time
+            cache[w.name] = (x, oracle.allreduce(wl.as_u16(x), w.block)["out"][0].copy())
+        return cache[w.name]
+    return get
+
+
 @pytest.mark.parametrize("variant", VARIANTS)
-@pytest.mark.parametrize("w", [wl.C2, wl.C3, wl.C5], ids=lambda w: w.name)
-def test_full_size_sampled(gu, w, variant):
-    """Full-size configs in the launch configuration the bench times (ping-pong workspace):
-    outputs of sampled blocks bit for bit, plus properties that hold at any size."""
+@pytest.mark.parametrize("w", [wl.C2, wl.C3], ids=lambda w: w.name)
+def test_full_size_every_word(gu, w, variant, full_size_expected):
+    """Configs 2 and 3 at full size, in the launch configuration the bench times (no trace):
+    EVERY output word of every rank against the oracle's evaluation of the whole tensor."""
+    x, exp = full_size_expected(w)
+    out, ws = gu.run_sim(x, w.block, keep_trace=False, variant=variant)
+    exp_dev = torch.from_numpy(exp.view(np.int16)).cuda()
+    for r in range(w.nranks):
+        same = torch.equal(out[r].view(torch.int16), exp_dev)
+        if not same:
+            gu.assert_same_words(out[r], exp, f"{variant} {w.name} rank {r}")
+    if variant == "steps":
+        _check_last_messages(ws, w)
+
+
+def _check_last_messages(ws, w):
+    # the last two messages of every shard are still in the workspace: codes within +-127
+    # and, per block, scale 0 or at least one |code| == 127
+    sc, co = eq.trace_views(ws.u8, w.nranks, w.count, w.block, keep_trace=False)
+    assert int(co.min()) >= -127
+    amax = co.view(2 * w.nranks, -1, w.block).abs().amax(dim=2)
+    assert bool(((amax == 127) | (sc == 0)).all())
+    assert bool(((sc != 0) | (amax == 0)).all())
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_stress_config_full_size_sampled(gu, variant):
+    """Config 5 at full size (64 ranks x 16 Mi elements: the oracle needs minutes for all of it):
+    300 sampled blocks of every shard bit for bit, plus properties that hold at any size."""
+    w = wl.C5
     x = wl.make_inputs(w, device="cuda")
     out, ws = gu.run_sim(x, w.block, keep_trace=False, variant=variant)
     for r in range(1, w.nranks):
         assert torch.equal(out[0].view(torch.int16), out[r].view(torch.int16)), "outputs differ across ranks"
     bps = w.count // w.nranks // w.block
-    picks = gu.sample_blocks(w.nranks, bps, 24, seed=1)
+    picks = gu.sample_blocks(w.nranks, bps, 300, seed=1)
     exp = gu.oracle_out_on_samples(x, picks, w.block)
     got = gu.gather_blocks(out, picks, w.block)
     gu.assert_same_words(got, exp, "sampled outputs")
     if variant == "steps":
-        # the last two messages of every shard are still in the workspace: codes within +-127
-        # and, per block, scale 0 or at least one |code| == 127
-        sc, co = eq.trace_views(ws.u8, w.nranks, w.count, w.block, keep_trace=False)
-        assert int(co.min()) >= -127
-        amax = co.view(2 * w.nranks, -1, w.block).abs().amax(dim=2)
-        assert bool(((amax == 127) | (sc == 0)).all())
-        assert bool(((sc != 0) | (amax == 0)).all())
+        _check_last_messages(ws, w)
 
 
 @pytest.mark.parametrize("nranks,count", [(1, 4096), (2, 2 * 4096 + 32), (4, 65536), (7, 7 * 16 * 301), (64, 64 * 4096)])
@@ -266,23 +301,6 @@ def test_sweep_points_large_sampled(gu, nranks, block, dist, nbytes):
     torch.cuda.empty_cache()
 
 
-def test_host_pipeline_matches_device_path(gu):
-    """The host-buffer front end (pinned memory in, pinned memory out, overlapped copies) returns
-    the same bits as the device-resident call, for several submissions in flight."""
-    from paper_2506_17615_b200.host_api import HostPipeline
-    w = wl.Workload("t", 4, 4 * 256 * 40, 256, "normal", seed=1)
-    pipe = HostPipeline(w.nranks, w.count, w.block)
-    xs = [wl.make_inputs(wl.Workload("t", 4, w.count, 256, "normal", seed=s)) for s in range(5)]
-    h_in = [x.pin_memory() for x in xs]
-    h_out = [torch.empty_like(x).pin_memory() for x in xs]
-    for i in range(5):
-        pipe.submit(h_in[i], h_out[i])
-    pipe.wait()
-    for i in range(5):
-        exp = oracle.allreduce(wl.as_u16(xs[i]), 256)["out"]
-        gu.assert_same_words(h_out[i], exp, f"submission {i}")
-
-
 def _random_cases(n, seed):
     rng = np.random.default_rng(seed)
     cases = []
@@ -304,26 +322,72 @@ def test_randomized_shapes_and_value_ranges(gu, nranks, block, bps, kind, seed):
     _compare_full(gu, x, block)
 
 
-def test_pipelined_fifo_holds_the_last_messages_of_each_warp(gu):
-    """Without a trace the pipelined schedule sends every hop message through a two-record staging
-    FIFO per warp.  With at most one tile per warp, warp w's FIFO must hold, on return, the last
-    two messages (events N-2 and N-1) of tile w, as 544-byte records: metadata sector, then codes."""
-    n, block, bps = 4, 128, 8                      # shard = 1024 elements = 2 tiles; 8 tiles in all
-    count = n * bps * block
-    x = wl.make_inputs(wl.Workload("t", n, count, block, "normal", seed=77))
-    res = oracle.allreduce(wl.as_u16(x), block, trace=True)
-    _, ws = gu.run_sim(x.cuda(), block, keep_trace=False, variant="pipelined")
-    fifo = ws.u8.cpu().numpy()
-    shard, per_tile = count // n, 512 // block
-    for tile in range(n * 2):
-        k, t = divmod(tile, 2)
-        for j in (n - 2, n - 1):
-            rec = fifo[tile * 1088 + (j & 1) * 544: tile * 1088 + (j & 1) * 544 + 544]
-            hdr = rec[:32].view(np.float32)
-            exp_sc = res["scales"][k, j, t * per_tile:(t + 1) * per_tile]
-            assert np.array_equal(hdr[:per_tile].view(np.uint32), exp_sc.view(np.uint32)), (tile, j)
-            assert not hdr[per_tile:].any()
-            assert np.array_equal(rec[32:].view(np.int8), res["codes"][k, j, t * 512:(t + 1) * 512]), (tile, j)
+def test_chain_fused_form_leaves_its_workspace_alone(gu):
+    """Without a trace the single-launch schedule keeps every hop message in registers: the
+    (token) workspace must come back untouched."""
+    n, block = 4, 128
+    count = n * 8 * block
+    x = wl.make_inputs(wl.Workload("t", n, count, block, "normal", seed=77)).cuda()
+    wb = eq.allreduce_sim_pipelined_workspace_bytes(n, count, block, False)
+    assert wb == binding.PIPELINE_MIN_WORKSPACE_BYTES
+    ws = torch.full((4096,), 0x5A, dtype=torch.uint8, device="cuda")
+    out = torch.empty_like(x)
+    eq.allreduce_sim_pipelined([x[r] for r in range(n)], [out[r] for r in range(n)], n, count, block, ws, wb, False,
+                               gu.stream_handle())
+    torch.cuda.synchronize()
+    assert bool((ws == 0x5A).all())
+    gu.assert_same_words(out, oracle.allreduce(wl.as_u16(x), block)["out"], "chain-fused outputs")
+
+
+@pytest.mark.parametrize("pinned", (True, False))
+@pytest.mark.parametrize("in_place", (False, True))
+def test_host_buffer_entry_matches_oracle(gu, pinned, in_place):
+    """equarx_allreduce_sim_host: host tensors in, host tensors out, copies issued by the library
+    on the caller's stream; two calls back to back on two streams with two staging buffers."""
+    n, block = 8, 256
+    count = n * block * 37
+    xs = [wl.make_inputs(wl.Workload("t", n, count, block, "normal", seed=s)) for s in (3, 4)]
+    exp = [oracle.allreduce(wl.as_u16(x), block)["out"] for x in xs]
+    h_in = [x.clone().pin_memory() if pinned else x.clone() for x in xs]
+    h_out = h_in if in_place else [torch.zeros_like(x).pin_memory() if pinned else torch.zeros_like(x) for x in xs]
+    sb = eq.allreduce_sim_host_staging_bytes(n, count)
+    stage = [gu.Guarded(sb) for _ in xs]
+    streams = [torch.cuda.Stream() for _ in xs]
+    warm = torch.zeros((n, count), dtype=torch.bfloat16).pin_memory()
+    eq.allreduce_sim_host([warm[r] for r in range(n)], [warm[r] for r in range(n)], n, count, block, stage[0], sb,
+                          streams[0].cuda_stream)        # first use loads the kernel's code onto the device
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    for i in range(2):
+        eq.allreduce_sim_host([h_in[i][r] for r in range(n)], [h_out[i][r] for r in range(n)], n, count, block,
+                              stage[i], sb, streams[i].cuda_stream)
+    for st in streams:
+        st.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0, "the call changed the amount of free device memory"
+    for i in range(2):
+        stage[i].check()
+        gu.assert_same_words(h_out[i], exp[i], f"host entry, call {i}")
+        gu.assert_same_words(stage[i].view(torch.bfloat16).view(n, count), exp[i], "staging holds the reduced tensors")
+
+
+def test_step_schedule_reuses_its_message_slots_without_stale_reads(gu):
+    """The launch-per-step schedule without a trace reuses its ping-pong message slots every two
+    steps and every call, under programmatic dependent launch.  Sixty calls back to back on one
+    stream, each on different data, must each give the bits of a traced run of the same data."""
+    n, block = 8, 256
+    count = n * block * 96
+    xs = [wl.make_inputs(wl.Workload("t", n, count, block, "normal", seed=200 + i)).cuda() for i in range(6)]
+    refs = [gu.run_sim(x, block, keep_trace=True)[0] for x in xs]
+    wb = eq.allreduce_sim_workspace_bytes(n, count, block, False)
+    ws = torch.empty(wb, dtype=torch.uint8, device="cuda")
+    outs = [torch.empty_like(xs[0]) for _ in range(60)]
+    s = gu.stream_handle()
+    for i in range(60):
+        x = xs[i % 6]
+        eq.allreduce_sim([x[r] for r in range(n)], [outs[i][r] for r in range(n)], n, count, block, ws, wb, False, s)
+    torch.cuda.synchronize()
+    for i in range(60):
+        assert torch.equal(outs[i].view(torch.int16), refs[i % 6].view(torch.int16)), f"call {i}"
 
 
 @pytest.mark.parametrize("nranks", (4, 8, 16))

@@ -7,11 +7,14 @@ cudaMalloc.  For them the library carries a fixed 16 MiB workspace of its own.
 This test calls that entry point through the C ABI twice in a row (the second
 call finds the first call's messages still in the shared workspace and must not
 be disturbed by them) and requires the same bits as equarx_allreduce_sim with a
-caller-provided workspace.  It is collected last on purpose.
+caller-provided workspace, and as the CPU oracle.  It also checks the claim in the
+entry point's purpose: the amount of free device memory is the same before and
+after the calls.  It is collected last on purpose.
 """
 import pytest
 import torch
 
+import oracle
 import paper_2506_17615_b200 as eq
 from paper_2506_17615_b200 import binding, workloads as wl
 
@@ -46,7 +49,47 @@ def test_static_workspace_matches_caller_workspace_twice_in_a_row():
         exp = _reference(x, block)
         assert torch.equal(got.view(torch.int16), exp.view(torch.int16))
     # and once more with the first problem: stale messages of another shape are in the array now
-    assert torch.equal(_static(first, 256).view(torch.int16), _reference(first, 256).view(torch.int16))
+    again = _static(first, 256)
+    assert torch.equal(again.view(torch.int16), _reference(first, 256).view(torch.int16))
+    # first hand: the oracle's bits
+    exp = oracle.allreduce(wl.as_u16(first), 256)["out"]
+    assert (wl.as_u16(again) == exp).all()
+
+
+def test_static_entry_allocates_no_device_memory():
+    x = wl.make_inputs(wl.Workload("a", 8, 8 * 256 * 150, 256, "normal", seed=23)).cuda()
+    n, count = x.shape
+    out = torch.empty_like(x)
+    ins, outs = [x[r] for r in range(n)], [out[r] for r in range(n)]
+    s = torch.cuda.current_stream().cuda_stream
+    eq.allreduce_sim_static(ins, outs, n, count, 256, s)       # set-up call: address look-up, code loading
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    reserved_before = torch.cuda.memory_reserved()
+    for _ in range(3):
+        eq.allreduce_sim_static(ins, outs, n, count, 256, s)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before
+    assert torch.cuda.memory_reserved() == reserved_before
+
+
+def test_static_entry_rejects_bad_tables_like_the_other_entry():
+    x = torch.zeros((4, 4 * 256), dtype=torch.bfloat16, device="cuda")
+    out = torch.empty_like(x)
+    ins, outs = [x[r] for r in range(4)], [out[r] for r in range(4)]
+    s = torch.cuda.current_stream().cuda_stream
+
+    def status(i, o):
+        with pytest.raises(eq.EquarxError) as err:
+            eq.allreduce_sim_static(i, o, 4, 4 * 256, 256, s)
+        return err.value.status
+
+    assert status(ins[:3] + [None], outs) == binding.ERR_NULL
+    assert status(ins, [outs[1]] + outs[1:]) == binding.ERR_ALIAS
+    assert status(ins, [ins[2]] + outs[1:]) == binding.ERR_ALIAS
+    assert status(ins, [outs[0].data_ptr() + 16] + outs[1:]) == binding.ERR_ALIGN
+    eq.allreduce_sim_static(ins, ins, 4, 4 * 256, 256, s)      # in place is allowed
+    torch.cuda.synchronize()
 
 
 def test_static_workspace_holds_the_largest_documented_case_and_rejects_more():
