@@ -303,6 +303,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the flavours and the bf16 comparator")
+    ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_SECONDS,
+                    help="GPU time to measure per schedule (trains of --steps steps are repeated); "
+                         "0 for profiling runs: three trains only")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -373,10 +376,13 @@ def main():
     windows = []
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
-    def timed(step_fn, steps, min_seconds=MIN_TIMED_SECONDS, max_trains=400):
+    def timed(step_fn, steps, min_seconds=None, max_trains=400):
         """Trains of exactly `steps` steps between CUDA events on the launching stream, each bracketed
         by a barrier + synchronize on both sides and reduced to the max over ranks; repeated until
         min_seconds of GPU time has been measured.  Returns (median ms per step, trains)."""
+        if min_seconds is None:
+            min_seconds = args.min_seconds
+        min_seconds = min(min_seconds, args.min_seconds)
         for i in range(args.warmup):
             step_fn(i)
         trains, total = [], 0.0
@@ -425,7 +431,7 @@ def main():
                    for _ in range(reps)] for t_ in ktrains}
     h0 = time.perf_counter()
     passes = 0
-    while passes < 3 or (time.perf_counter() - h0 < 0.5 and passes < 2000):   # also gives the clock sampler load
+    while passes < 3 or (time.perf_counter() - h0 < args.min_seconds and passes < 2000):   # also gives the clock sampler load
         for i in range(reps):
             for name, first, last, repeat, _ in ktrains:
                 a, b = evs[name][i]

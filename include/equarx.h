@@ -327,6 +327,59 @@ int equarx_allreduce_sim_static(const void *const *in_bf16, void *const *out_bf1
                                 int nranks, size_t count, int block,
                                 equarx_stream_t stream);
 
+/*
+ * The quantized ring AllReduce with one rank per device: the setting of Section 3
+ * (Fig. 1) and Section 3.1 (Fig. 2: metadata first, microshards pipelined so that
+ * transfers overlap the dequantize / add / quantize work).  Each rank runs ONE
+ * persistent kernel that performs all nranks ring steps and the all-gather.  A
+ * microshard is a tile of 512 elements and its message one 544-byte record (layout as
+ * for equarx_allreduce_sim).  The sending rank stores the record directly into the
+ * RECEIVING rank's mailbox (peer memory: NVLink when the ranks are on different GPUs)
+ * and then releases a per-tile flag; the receiving warp polls that flag.  The last
+ * reduce-scatter step stores the all-gather message of the rank's own shard into every
+ * rank's mailbox, and every rank dequantizes the nranks messages it received.  Ring
+ * direction, shard order and arithmetic are those of equarx_allreduce_sim, so the
+ * outputs and every message are identical to it bit for bit.
+ *
+ * A call hosts the consecutive ranks rank_first .. rank_first + ranks_here - 1 on the
+ * current device, in one cooperative launch (all its CTAs are resident at once).
+ * ranks_here = 1 is the multi-GPU case: one process and one call per GPU, all with
+ * the same epoch.  ranks_here = nranks runs the whole ring on a single GPU.
+ *
+ *   in_bf16[i], out_bf16[i] : HOST arrays of ranks_here DEVICE pointers: tensors of
+ *                 rank rank_first + i (count bf16 words each; out may equal in)
+ *   mailboxes   : HOST array of nranks DEVICE-addressable pointers, mailbox of every
+ *                 rank of the ring, own ranks included; a peer's mailbox is its
+ *                 allocation mapped into this process (CUDA IPC or any other
+ *                 peer mapping).  Each is equarx_ring_mailbox_bytes() bytes, 32-byte
+ *                 aligned, and must be zeroed ONCE before its first use.
+ *                 Layout: slots 0..nranks-2 hold the message received at ring step
+ *                 slot+1, slots nranks-1..2*nranks-2 the all-gather message of shard
+ *                 slot-(nranks-1); a slot is ceil(count/nranks/512) records; then one
+ *                 uint32 flag per (slot, tile), slot-major.
+ *   epoch       : >= 1, the same on every rank of one AllReduce, and larger than in
+ *                 any earlier call that used these mailboxes (a flag equal to the
+ *                 epoch marks a complete record, so nothing is cleared between calls).
+ *                 Calls that share mailboxes must be ordered on each rank's stream.
+ *   timeout_ns  : longest wait for one message; 0 selects 1 second.  A wait that runs
+ *                 out, or that sees another warp's failure, makes the warp record
+ *                 {EQUARX_RING_TIMEOUT, rank, step, tile} in `status` (first failure
+ *                 only) and leave; the kernel always terminates, never traps.  step is
+ *                 the ring step, or nranks + shard for an all-gather message.
+ *   status      : DEVICE memory, 4 x uint32, 16-byte aligned, zeroed by the caller;
+ *                 read it after synchronising: code 0 means every message arrived.
+ * Returns EQUARX_ERR_CUDA if the cooperative launch is refused (for example more hosted
+ * ranks than CTAs that fit on the device).
+ * Not exercised on more than one GPU; the ranks_here = nranks form is what the tests run.
+ */
+#define EQUARX_RING_OK 0u
+#define EQUARX_RING_TIMEOUT 1u
+size_t equarx_ring_mailbox_bytes(int nranks, size_t count, int block);
+int equarx_ring_allreduce(const void *const *in_bf16, void *const *out_bf16,
+                          int rank_first, int ranks_here, int nranks, size_t count, int block,
+                          void *const *mailboxes, uint32_t epoch, uint64_t timeout_ns,
+                          uint32_t *status, equarx_stream_t stream);
+
 /* Static, human-readable name of a status. */
 const char *equarx_status_string(int status);
 

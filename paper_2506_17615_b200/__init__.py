@@ -36,6 +36,8 @@ _BINDING_NAMES = (
     "last_cuda_error",
     "lib",
     "quantize_blocks",
+    "ring_allreduce",
+    "ring_mailbox_bytes",
     "rs_step_dequant_add_requant",
     "status_string",
     "trace_views",

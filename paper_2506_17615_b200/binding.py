@@ -27,6 +27,8 @@ EXPORTS = (
     "equarx_allreduce_sim_pipelined",
     "equarx_allreduce_sim_pipelined_workspace_bytes",
     "equarx_allreduce_sim_host",
+    "equarx_ring_allreduce",
+    "equarx_ring_mailbox_bytes",
     "equarx_allreduce_sim_host_staging_bytes",
     "equarx_allreduce_sim_range",
     "equarx_allreduce_sim_static",
@@ -60,6 +62,9 @@ def _load():
     lib.equarx_allreduce_sim_host.argtypes = [vp, vp, ci, sz, ci, vp, sz, vp]
     lib.equarx_allreduce_sim_host_staging_bytes.argtypes = [ci, sz]
     lib.equarx_allreduce_sim_host_staging_bytes.restype = sz
+    lib.equarx_ring_mailbox_bytes.argtypes = [ci, sz, ci]
+    lib.equarx_ring_mailbox_bytes.restype = sz
+    lib.equarx_ring_allreduce.argtypes = [vp, vp, ci, ci, ci, sz, ci, vp, ctypes.c_uint32, ctypes.c_uint64, vp, vp]
     lib.equarx_allreduce_sim_flavour.argtypes = [vp, vp, ci, sz, ci, ci, vp, sz, ci, vp]
     lib.equarx_allreduce_sim_flavour_workspace_bytes.argtypes = [ci, sz, ci, ci, ci]
     lib.equarx_allreduce_sim_flavour_workspace_bytes.restype = sz
@@ -154,6 +159,22 @@ def allreduce_sim_host(host_in, host_out, nranks, count, block, staging, staging
     _check(lib.equarx_allreduce_sim_host(_table(host_in), _table(host_out), nranks, count, block, _ptr(staging),
                                          staging_bytes, _ptr(stream)),
            "equarx_allreduce_sim_host")
+
+
+RING_OK, RING_TIMEOUT = 0, 1
+
+
+def ring_mailbox_bytes(nranks, count, block):
+    return lib.equarx_ring_mailbox_bytes(nranks, count, block)
+
+
+def ring_allreduce(in_bf16, out_bf16, rank_first, ranks_here, nranks, count, block, mailboxes, epoch, timeout_ns,
+                   status, stream=0):
+    """equarx_ring_allreduce: the ranks rank_first .. rank_first+ranks_here-1 of the ring on the current
+    device; `mailboxes` lists every rank's mailbox, `status` is 4 zeroed uint32 words on the device."""
+    _check(lib.equarx_ring_allreduce(_table(in_bf16), _table(out_bf16), rank_first, ranks_here, nranks, count, block,
+                                     _table(mailboxes), epoch, timeout_ns, _ptr(status), _ptr(stream)),
+           "equarx_ring_allreduce")
 
 
 def allreduce_sim_flavour_workspace_bytes(nranks, count, block, flavour, keep_trace=False):

@@ -580,6 +580,98 @@ int equarx_allreduce_sim_flavour(const void* const* in_bf16, void* const* out_bf
     return EQUARX_OK;
 }
 
+size_t equarx_ring_mailbox_bytes(int nranks, size_t count, int block) {
+    if (check_sim_shape(nranks, count, block) != EQUARX_OK) return 0;
+    const size_t N = size_t(nranks);
+    const size_t tiles = (count / N + kTileElems - 1) / kTileElems;
+    const size_t slots = 2 * N - 1;
+    const size_t bytes = slots * tiles * size_t(kRecordBytes) + slots * tiles * sizeof(uint32_t);
+    return (bytes + 255) / 256 * 256;
+}
+
+int equarx_ring_allreduce(const void* const* in_bf16, void* const* out_bf16, int rank_first, int ranks_here,
+                          int nranks, size_t count, int block, void* const* mailboxes, uint32_t epoch,
+                          uint64_t timeout_ns, uint32_t* status, equarx_stream_t stream) {
+    if (int st = check_sim_shape(nranks, count, block)) return st;
+    if (rank_first < 0 || ranks_here < 1 || rank_first + ranks_here > nranks) return EQUARX_ERR_NRANKS;
+    if (epoch == 0) return EQUARX_ERR_COUNT;
+    if (!in_bf16 || !out_bf16 || !mailboxes || !status) return EQUARX_ERR_NULL;
+    const size_t bytes = 2 * count, box_bytes = equarx_ring_mailbox_bytes(nranks, count, block);
+    for (int i = 0; i < ranks_here; ++i)
+        if (!in_bf16[i] || !out_bf16[i]) return EQUARX_ERR_NULL;
+    for (int q = 0; q < nranks; ++q)
+        if (!mailboxes[q]) return EQUARX_ERR_NULL;
+    if (!aligned(status, 16)) return EQUARX_ERR_ALIGN;
+    for (int i = 0; i < ranks_here; ++i)
+        if (!aligned(in_bf16[i], 32) || !aligned(out_bf16[i], 32)) return EQUARX_ERR_ALIGN;
+    for (int q = 0; q < nranks; ++q)
+        if (!aligned(mailboxes[q], 32)) return EQUARX_ERR_ALIGN;
+    for (int i = 0; i < ranks_here; ++i) {
+        for (int j = 0; j < ranks_here; ++j) {
+            if (j != i && overlap(out_bf16[i], bytes, out_bf16[j], bytes)) return EQUARX_ERR_ALIAS;
+            if (overlap(out_bf16[i], bytes, in_bf16[j], bytes) && !(j == i && out_bf16[i] == in_bf16[j]))
+                return EQUARX_ERR_ALIAS;
+        }
+        for (int q = 0; q < nranks; ++q)
+            if (overlap(mailboxes[q], box_bytes, in_bf16[i], bytes) || overlap(mailboxes[q], box_bytes, out_bf16[i], bytes))
+                return EQUARX_ERR_ALIAS;
+    }
+    for (int q = 0; q < nranks; ++q)
+        for (int p = q + 1; p < nranks; ++p)
+            if (overlap(mailboxes[q], box_bytes, mailboxes[p], box_bytes)) return EQUARX_ERR_ALIAS;
+
+    const uint32_t N = uint32_t(nranks);
+    RingArgs a = {};
+    a.neg_zero = -0.0f;
+    for (int i = 0; i < ranks_here; ++i) {
+        a.in[i] = in_bf16[i];
+        a.out[i] = out_bf16[i];
+    }
+    for (uint32_t q = 0; q < N; ++q) a.mailbox[q] = static_cast<char*>(mailboxes[q]);
+    a.status = status;
+    a.shard = count / N;
+    a.tiles_per_shard = (a.shard + kTileElems - 1) / kTileElems;
+    a.timeout_ns = timeout_ns ? timeout_ns : 1000000000ull;
+    a.nranks = N;
+    a.rank_first = uint32_t(rank_first);
+    a.ranks_here = uint32_t(ranks_here);
+    a.epoch = epoch;
+
+    const void* kernel = nullptr;
+    switch (block) {
+        case 64: kernel = reinterpret_cast<const void*>(ring_rank_kernel<4>); break;
+        case 128: kernel = reinterpret_cast<const void*>(ring_rank_kernel<8>); break;
+        case 256: kernel = reinterpret_cast<const void*>(ring_rank_kernel<16>); break;
+        default: kernel = reinterpret_cast<const void*>(ring_rank_kernel<32>); break;
+    }
+    auto failed = [](cudaError_t e) {
+        g_last_cuda_error = int(e);
+        (void)cudaGetLastError();
+        return EQUARX_ERR_CUDA;
+    };
+    int dev = 0, sms = 0, occ = 0, coop = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kRingThreads, 0);
+    if (e != cudaSuccess) return failed(e);
+    if (sms < 1 || occ < 1 || !coop) return failed(cudaErrorCooperativeLaunchTooLarge);
+    // every hosted rank gets the same number of CTAs and all of them must be resident at once
+    const uint64_t resident = uint64_t(sms) * uint64_t(occ);
+    const uint64_t wpc = kRingThreads / 32;
+    uint64_t per_rank = resident / uint64_t(ranks_here);
+    per_rank = std::min<uint64_t>(per_rank, (a.tiles_per_shard + wpc - 1) / wpc);
+    if (per_rank < 1) return failed(cudaErrorCooperativeLaunchTooLarge);
+    a.ctas_per_rank = uint32_t(per_rank);
+    void* params[1] = {&a};
+    e = injected_launch_error();
+    if (e == cudaSuccess)
+        e = cudaLaunchCooperativeKernel(kernel, dim3(unsigned(per_rank * uint64_t(ranks_here))), dim3(kRingThreads),
+                                        params, 0, stream);
+    if (e != cudaSuccess) return failed(e);
+    return EQUARX_OK;
+}
+
 size_t equarx_allreduce_sim_bf16_workspace_bytes(int nranks, size_t count) {
     if (nranks < 1 || nranks > EQUARX_MAX_RANKS) return 0;
     if (count == 0 || count > kMaxCount || count % (size_t(nranks) * kLaneElems) != 0) return 0;

@@ -1104,6 +1104,193 @@ __global__ void __launch_bounds__(kPipeThreads) flavour_fused_kernel(const __gri
     }
 }
 
+// ---------------------------------------------------------------- the ring across devices
+// The paper's own setting (Section 3, Fig. 1; Section 3.1, Fig. 2): one rank per device, every
+// reduce-scatter step a send to the right neighbour and a receive from the left one, metadata
+// ahead of the payload, microshards pipelined.  A rank's kernel is ONE persistent launch that runs
+// all N ring steps and the all-gather; a microshard is a 512-element tile, its message one
+// 544-byte record.  The sender stores the record straight into the RECEIVER's mailbox (plain
+// 16-byte stores: over NVLink when the mailbox lives on another GPU) and then releases a per-tile
+// flag word; the receiver's warp for that tile polls the flag with a BOUNDED wait.  Tiles advance
+// independently, so a tile's hop overlaps the transfers of all other tiles.  The last
+// reduce-scatter step stores the all-gather message of the rank's own shard into every rank's
+// mailbox (each peer is reachable at full bandwidth through the switch), and every rank
+// dequantizes what it received.  No bulk-tensor copy and no multicast of any kind is used.
+//
+// Mailbox of a rank (device memory, zeroed once before its first use):
+//   slots 0..N-2   : the message received at ring step s = slot + 1 (tiles_per_shard records)
+//   slots N-1..2N-2: the all-gather message of shard k = slot - (N-1)
+//   then one 32-bit flag per (slot, tile); a flag equal to the call's epoch means "record complete".
+// Epochs grow from call to call, so nothing is cleared between calls.  A slot is only rewritten
+// after its reader is done with it: rank r's call e returns only once it holds the all-gather
+// record of every tile of every shard, and rank q produces tile t of its all-gather message after
+// its last read of tile t of any reduce-scatter slot (one warp owns a tile index through all steps).
+//
+// A launch can host several consecutive ranks (ranks_here > 1): their CTAs are co-resident (the
+// launch is cooperative) and exchange through the same mailboxes, which is how the whole ring runs
+// and is checked on a single GPU.
+constexpr int kRingThreads = 128;
+constexpr uint32_t kRingOk = 0, kRingTimeout = 1;
+
+struct RingArgs {
+    const void* in[kMaxRanks];       // input tensor of hosted rank rank_first + i
+    void* out[kMaxRanks];            // output tensor of hosted rank rank_first + i
+    char* mailbox[kMaxRanks];        // mailbox of EVERY rank of the ring, as addressable from this device
+    uint32_t* status;                // {code, rank, step, tile}: first failure of this launch, else untouched
+    uint64_t shard;
+    uint64_t tiles_per_shard;
+    uint64_t timeout_ns;             // longest wait for one message
+    uint32_t nranks, rank_first, ranks_here, ctas_per_rank;
+    uint32_t epoch;
+    float neg_zero;
+};
+
+__device__ __forceinline__ uint32_t ld_acquire_sys_u32(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_sys_u32(uint32_t* p, uint32_t v) {
+    asm volatile("st.release.sys.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+// data written by another device (or another SM): strong loads, never served from a stale L1 line
+__device__ __forceinline__ uint4 ld_relaxed_sys_128(const void* p) {
+    uint4 r;
+    asm volatile("ld.relaxed.sys.global.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p) : "memory");
+    return r;
+}
+__device__ __forceinline__ float ld_relaxed_sys_f32(const float* p) {
+    float r;
+    asm volatile("ld.relaxed.sys.global.f32 %0, [%1];" : "=f"(r) : "l"(p) : "memory");
+    return r;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Lane 0 polls the flag until it holds `epoch` or the time limit passes; the verdict is
+// broadcast, and the acquire orders the record loads of every lane after the flag.
+// A wait also gives up as soon as another warp of this launch has recorded a failure.
+__device__ __forceinline__ bool ring_wait(const uint32_t* flag, uint32_t epoch, uint64_t timeout_ns,
+                                          const uint32_t* status, uint32_t lane) {
+    uint32_t ok = 1;
+    if (lane == 0) {
+        if (ld_acquire_sys_u32(flag) != epoch) {
+            const uint64_t t0 = global_timer_ns();
+            for (uint32_t spins = 1;; ++spins) {
+                if (ld_acquire_sys_u32(flag) == epoch) break;
+                if ((spins & 15u) == 0 &&
+                    (global_timer_ns() - t0 > timeout_ns || *reinterpret_cast<const volatile uint32_t*>(status) != 0)) {
+                    ok = 0;
+                    break;
+                }
+                __nanosleep(64);
+            }
+        }
+    }
+    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+    return ok != 0;
+}
+
+template <int LPB>
+__global__ void __launch_bounds__(kRingThreads) ring_rank_kernel(const __grid_constant__ RingArgs a) {
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t N = a.nranks;
+    const uint32_t local = blockIdx.x / a.ctas_per_rank;             // hosted rank index
+    const uint32_t r = a.rank_first + local;                          // this CTA's rank
+    const uint32_t right = r + 1 == N ? 0 : r + 1;
+    const uint64_t warps = (uint64_t)a.ctas_per_rank * (kRingThreads / 32);
+    const uint64_t warp = (uint64_t)(blockIdx.x - local * a.ctas_per_rank) * (kRingThreads / 32) + (threadIdx.x >> 5);
+    const uint64_t T = a.tiles_per_shard;
+    const uint64_t groups = a.shard >> 4;
+    const uint64_t slot_bytes = T * kRecordBytes;
+    const uint64_t flags_at = (uint64_t)(2 * N - 1) * slot_bytes;     // byte offset of the flag words
+    const char* const x_rank = static_cast<const char*>(a.in[local]);
+    char* const my_box = a.mailbox[r];
+    auto flag_of = [&](char* box, uint32_t slot, uint64_t t) {
+        return reinterpret_cast<uint32_t*>(box + flags_at) + (uint64_t)slot * T + t;
+    };
+    auto fail = [&](uint32_t step, uint64_t t) {                      // first failure wins; then this warp leaves
+        if (lane == 0 && atomicCAS(a.status, kRingOk, kRingTimeout) == kRingOk) {
+            a.status[1] = r;
+            a.status[2] = step;
+            a.status[3] = (uint32_t)t;
+        }
+    };
+
+    // ---- reduce-scatter: step s sends shard (r - 1 - s) mod N
+    for (uint32_t s = 0; s < N; ++s) {
+        const uint32_t k = (r + 2 * N - 1 - s) % N;
+        for (uint64_t t = warp; t < T; t += warps) {
+            const bool active = t * 32 + lane < groups;
+            Vec8 xw = {};
+            if (active) xw = ld_coherent_256(x_rank + ((uint64_t)k * a.shard + (t * 32 + lane) * 16) * 2);   // in place is allowed
+            float v[16];
+            widen_bf16x16(xw, v);
+            if (s > 0) {                                              // the message received at this step
+                if (!ring_wait(flag_of(my_box, s - 1, t), a.epoch, a.timeout_ns, a.status, lane)) {
+                    fail(s, t);
+                    return;
+                }
+                const char* rec = my_box + (uint64_t)(s - 1) * slot_bytes + t * kRecordBytes;
+                uint4 c = make_uint4(0, 0, 0, 0);
+                float sc = 0.0f;
+                if (active) {
+                    c = ld_relaxed_sys_128(rec + kRecordHeader + lane * 16);
+                    sc = ld_relaxed_sys_f32(reinterpret_cast<const float*>(rec) + lane / LPB);
+                }
+                dequant_add_x16(c, sc, v);
+            }
+            uint4 codes;
+            float scale;
+            quantize_lane<LPB>(v, codes, scale, a.neg_zero);
+            float hdr = __shfl_sync(0xFFFFFFFFu, scale, (lane * LPB) & 31u);   // lanes 0..7: the metadata sector
+            if (lane >= 32u / LPB) hdr = 0.0f;
+            if (s + 1 < N) {
+                // to the right neighbour, as the message it receives at step s + 1
+                char* box = a.mailbox[right];
+                char* rec = box + (uint64_t)s * slot_bytes + t * kRecordBytes;
+                if (lane < 8) st_plain_f32(reinterpret_cast<float*>(rec) + lane, hdr);
+                if (active) st_plain_128(rec + kRecordHeader + lane * 16, codes);
+                __syncwarp();
+                if (lane == 0) st_release_sys_u32(flag_of(box, s, t), a.epoch);
+            } else {
+                // the reduced shard (k == r): its all-gather message goes to every rank
+                for (uint32_t q = 0; q < N; ++q) {
+                    char* box = a.mailbox[q];
+                    char* rec = box + (uint64_t)(N - 1 + k) * slot_bytes + t * kRecordBytes;
+                    if (lane < 8) st_plain_f32(reinterpret_cast<float*>(rec) + lane, hdr);
+                    if (active) st_plain_128(rec + kRecordHeader + lane * 16, codes);
+                }
+                __syncwarp();
+                if (lane == 0)
+                    for (uint32_t q = 0; q < N; ++q) st_release_sys_u32(flag_of(a.mailbox[q], N - 1 + k, t), a.epoch);
+            }
+        }
+    }
+
+    // ---- all-gather receive side: dequantize every shard's message into this rank's output
+    char* const out_rank = static_cast<char*>(a.out[local]);
+    for (uint32_t i = 0; i < N; ++i) {
+        const uint32_t k = (r + i) % N;                               // own shard first: it is already here
+        for (uint64_t t = warp; t < T; t += warps) {
+            if (!ring_wait(flag_of(my_box, N - 1 + k, t), a.epoch, a.timeout_ns, a.status, lane)) {
+                fail(N + k, t);
+                return;
+            }
+            if (t * 32 + lane >= groups) continue;
+            const char* rec = my_box + (uint64_t)(N - 1 + k) * slot_bytes + t * kRecordBytes;
+            const uint4 c = ld_relaxed_sys_128(rec + kRecordHeader + lane * 16);
+            const float sc = ld_relaxed_sys_f32(reinterpret_cast<const float*>(rec) + lane / LPB);
+            const Vec8 o = dequant_to_bf16x16(c, sc);
+            st_stream_256(out_rank + ((uint64_t)k * a.shard + (t * 32 + lane) * 16) * 2, o);
+        }
+    }
+}
+
 // Unquantized comparator hop: send = bf16_rne(f32(recv) + f32(local)).
 __global__ void __launch_bounds__(kThreads) bf16_step_kernel(const __grid_constant__ Bf16StepArgs a) {
     const uint32_t r = blockIdx.y;
