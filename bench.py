@@ -293,6 +293,82 @@ def roofline_entry(kernel, bytes_per_launch, ms_per_launch, peak, peak_src, traf
             "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
 
 
+def run_ring(args):
+    """--ring: the ring with one rank per GPU (equarx_ring_allreduce through PeerRing): every process
+    is one rank, messages go into the neighbours' mailboxes over peer memory.  The number of ranks is
+    the number of processes; each rank holds the workload's per-rank tensor.  Not exercised on more
+    than one GPU: every device-side wait is bounded, so a rank that cannot reach its peers reports
+    a time-out instead of hanging."""
+    import torch
+    import torch.distributed as dist
+    from paper_2506_17615_b200 import workloads as wl
+    from paper_2506_17615_b200.ring import PeerRing, RingTimeout
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29531")
+    # the process group carries IPC handles, barriers and the max only; no multimem/NVLS is used anywhere
+    dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+    base = workload_by_name(args.workload)
+    unit = _lcm(base.hidden, world * base.block) if base.hidden else world * base.block
+    count = max(unit, base.count // unit * unit)
+    w = wl.Workload(base.name + f"_ring{world}", world, count, base.block, base.dist, base.hidden, base.seed)
+    x = wl.make_rank(w, rank, device=dev)
+    out = torch.empty_like(x)
+    ring = PeerRing(count, w.block)
+    stream = torch.cuda.current_stream().cuda_stream
+    timeout_ns = 2_000_000_000
+
+    def barrier():
+        dist.barrier()
+        torch.cuda.synchronize()
+
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    failure = None
+    try:
+        for _ in range(args.warmup):
+            ring.allreduce(x, out, timeout_ns, stream)
+            ring.check()
+        trains, total = [], 0.0
+        while len(trains) < 3 or (total < args.min_seconds * 1e3 and len(trains) < 400):
+            barrier()
+            ev0.record()
+            for _ in range(args.steps):
+                ring.allreduce(x, out, timeout_ns, stream)
+            ev1.record()
+            torch.cuda.synchronize()
+            ring.check()
+            barrier()
+            ms = max_over_ranks(ev0.elapsed_time(ev1), world, dev)
+            trains.append(ms)
+            total += ms
+        ms_step = statistics.median(trains) / args.steps
+    except RingTimeout as exc:
+        failure = str(exc)
+        ms_step = float("nan")
+    if rank == 0:
+        peak, peak_src = hbm_peak()
+        in_bytes = 2 * count * world
+        wire = count * (1.0 + 4.0 / w.block) / world            # one shard's message
+        # per rank: N local shard reads, N-1 messages stored to the right neighbour and N to everybody's
+        # all-gather slot, as many read, N shard writes
+        link_bytes = (world - 1) * wire + (world - 1) * wire     # crossing NVLink, per rank and direction
+        line = {"metric": METRIC, "value": in_bytes / (ms_step * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {**base_config(w, 1), "parallelism": f"ring, one rank per GPU x{world}"},
+                "schedule": "equarx_ring_allreduce, ranks_here=1 (peer mailboxes, per-tile flags)",
+                "nvlink_bytes_per_rank_and_direction": link_bytes, "gpu_launches": args.steps,
+                "failure": failure, "note": "not exercised on more than one GPU"}
+        print(json.dumps(line))
+    if failure is None:
+        ring.close()
+    dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -303,6 +379,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the flavours and the bf16 comparator")
+    ap.add_argument("--ring", action="store_true",
+                    help="one rank of a real ring per process/GPU instead of independent replicas (opt-in)")
     ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_SECONDS,
                     help="GPU time to measure per schedule (trains of --steps steps are repeated); "
                          "0 for profiling runs: three trains only")
@@ -313,6 +391,9 @@ def main():
         args.steps = 1
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.ring:
+        run_ring(args)
         return
 
     import torch
@@ -467,7 +548,7 @@ def main():
                 "hop_traffic_bytes_per_launch": hop["bytes_per_element"] * count,
                 "hop_traffic_source": f"ncu, {hop['profile']}, scaled by elements"}
 
-    flavours, bf16_sim, ratios = {}, None, None
+    flavours, bf16_sim, ratios, ring_local = {}, None, None, None
     if not args.no_extras:
         # ---- the other flavours (semi-loop ring, stage selection, FP8), same workload, single launch
         wbf = eq.allreduce_sim_flavour_workspace_bytes(N, count, block, 7 if N % 2 == 0 else 6, False)
@@ -483,6 +564,25 @@ def main():
                             max(5, min(50, args.steps)), min_seconds=0.1)
             flavours[name] = {"ms_per_step": ms_f, "value": aggregate_value(in_bytes, ms_f, world), "unit": UNIT}
         del wsf
+
+        # ---- the ring with one rank per device, all ranks hosted by this GPU (mailboxes + per-tile flags)
+        from paper_2506_17615_b200.ring import LocalRing
+        lring = LocalRing(N, count, block, dev)
+
+        def step_ring(i):
+            lring.allreduce(ins[i % sets], outs[i % sets], 0, stream)
+
+        ms_r, _ = timed(step_ring, max(5, min(50, args.steps)), min_seconds=0.2)
+        lring.check()
+        wire = count * (1.0 + 4.0 / block)
+        ring_bytes = 4.0 * count * N + 2.0 * (N - 1) * wire + 2.0 * N * wire
+        ring_local = {"ms_per_step": ms_r, "value": aggregate_value(in_bytes, ms_r, world), "unit": UNIT,
+                      "schedule": "equarx_ring_allreduce, all ranks hosted by one cooperative launch",
+                      "bytes_per_launch": ring_bytes,
+                      "bytes_model": "inputs and outputs once; N-1 reduce-scatter messages per shard written and read "
+                                     "once; the all-gather message of every shard written to and read from N mailboxes",
+                      "frac": ring_bytes / (ms_r * 1e-3) / 1e9 / peak}
+        del lring
 
         # ---- unquantized comparator on the same GPU, same inputs, one launch per ring step
         wb16 = eq.allreduce_sim_bf16_workspace_bytes(N, count)
@@ -553,7 +653,7 @@ def main():
             "e2e": e2e, "gpu_launches": args.steps, "clocks": clocks,
             "roofline": roofline,
             "schedule": "chain-fused single launch (equarx_allreduce_sim_pipelined, keep_trace=0)",
-            "by_steps": by_steps, "flavours": flavours, "bf16_sim": bf16_sim,
+            "by_steps": by_steps, "ring_on_one_gpu": ring_local, "flavours": flavours, "bf16_sim": bf16_sim,
             "speedup_vs_bf16": ratios, "input_checksum": checksum,
             "pdl_between_step_launches": os.environ.get("EQUARX_PDL", "1") != "0",
         }

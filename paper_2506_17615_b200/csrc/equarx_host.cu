@@ -116,6 +116,23 @@ int launch_gather(int block, const GatherArgs& a, cudaStream_t stream, bool depe
     }
 }
 
+// Persistent grid of the single-launch kernels: a whole number of CTAs per SM (measured: a grid that
+// balances the warps' tile counts but loads the SMs unevenly is 2 % slower at 88 MB per rank and no
+// faster at 16 MB), the count per SM that needs the fewest rounds of tiles and, among those, the
+// smallest; never more CTAs than there are tiles to carry.
+inline uint64_t persistent_grid(uint64_t tiles, uint64_t warps_per_cta, int sms, int occ) {
+    uint64_t best = 0, best_rounds = ~uint64_t(0);
+    for (int c = 1; c <= occ; ++c) {
+        const uint64_t ctas = uint64_t(sms) * c, w = ctas * warps_per_cta;
+        const uint64_t rounds = (tiles + w - 1) / w;
+        if (rounds < best_rounds) {
+            best_rounds = rounds;
+            best = ctas;
+        }
+    }
+    return std::min<uint64_t>(best, (tiles + warps_per_cta - 1) / warps_per_cta);
+}
+
 // bytes of one message slot in the record layout: one 544-byte record per 512-element tile
 inline size_t slot_bytes(size_t shard) { return (shard + kTileElems - 1) / kTileElems * size_t(kRecordBytes); }
 
@@ -326,8 +343,10 @@ int equarx_allreduce_sim_range(const void* const* in_bf16, void* const* out_bf16
             a.out_slot[r] = slot_of(s, r);
             a.in_slot[r] = s ? slot_of(s - 1, (r + N - 1) % N) : 0;
         }
-        // only a launch that follows another launch of this call may overlap its predecessor
-        const int st = s == 0 ? launch_step<true, true>(block, a, N, stream, false)
+        // step 0 waits for the stream's earlier work before its first load, so it can always be a
+        // programmatic dependent; a later step loads its shard ahead of the wait and may only overlap
+        // a launch of this same call
+        const int st = s == 0 ? launch_step<true, true>(block, a, N, stream, true)
                               : launch_step<false, true>(block, a, N, stream, s > first);
         if (st) return st;
     }
@@ -370,18 +389,21 @@ int launch_pipelined(const void* const* in_bf16, void* const* out_bf16, int nran
     a.tiles_per_shard = (shard + kTileElems - 1) / kTileElems;
     a.nranks = N;
 
-    constexpr int D = EQX_FUSED_DEPTH;
+    constexpr int D = kFusedDepth;
+    // register budget of the chain-fused kernel: see chain_fused_kernel
+    const bool large = 2.0 * double(count) * double(nranks) > 200e6;
     const void* kernel = nullptr;
-#define EQX_PICK(L)                                                                                   \
-    kernel = keep_trace ? reinterpret_cast<const void*>(pipelined_kernel<L>)                          \
-             : quantized ? reinterpret_cast<const void*>(chain_fused_kernel<L, D, true>)              \
-                         : reinterpret_cast<const void*>(chain_fused_kernel<L, D, false>)
+#define EQX_FUSED(L, Q) (large ? reinterpret_cast<const void*>(chain_fused_kernel<L, D, Q, 16>) \
+                               : reinterpret_cast<const void*>(chain_fused_kernel<L, D, Q, 18>))
+#define EQX_PICK(L) \
+    kernel = keep_trace ? reinterpret_cast<const void*>(pipelined_kernel<L>) : quantized ? EQX_FUSED(L, true) : EQX_FUSED(L, false)
     switch (block) {
         case 64: EQX_PICK(4); break;
         case 128: EQX_PICK(8); break;
         case 256: EQX_PICK(16); break;
         default: EQX_PICK(32); break;
     }
+#undef EQX_FUSED
 #undef EQX_PICK
     // persistent grid: a whole number of CTAs per SM
     int dev = 0, sms = 0, occ = 0;
@@ -393,21 +415,7 @@ int launch_pipelined(const void* const* in_bf16, void* const* out_bf16, int nran
         (void)cudaGetLastError();
         return EQUARX_ERR_CUDA;
     }
-    // The kernel is bound by the latency of the per-tile chain, so a round (every warp carries one
-    // tile through the ring) costs about the same whatever the number of resident warps: take the
-    // CTA count per SM that needs the fewest rounds and, among those, the smallest one.
-    const uint64_t tiles = a.tiles_per_shard * N, wpc = kPipeThreads / 32;
-    uint64_t best_ctas = 0, best_rounds = ~uint64_t(0);
-    for (int c = 1; c <= occ; ++c) {
-        const uint64_t ctas = uint64_t(sms) * c, w = ctas * wpc;
-        const uint64_t rounds = (tiles + w - 1) / w;
-        if (rounds < best_rounds) {
-            best_rounds = rounds;
-            best_ctas = ctas;
-        }
-    }
-    const uint64_t max_needed = (tiles + wpc - 1) / wpc;
-    if (best_ctas > max_needed) best_ctas = max_needed;
+    const uint64_t best_ctas = persistent_grid(a.tiles_per_shard * N, kPipeThreads / 32, sms, occ);
 
     // programmatic dependent launch hides the launch latency behind the previous kernel's tail; the
     // kernel itself waits for that kernel to complete before its first memory access
@@ -550,16 +558,8 @@ int equarx_allreduce_sim_flavour(const void* const* in_bf16, void* const* out_bf
         (void)cudaGetLastError();
         return EQUARX_ERR_CUDA;
     }
-    const uint64_t tiles = a.tiles_per_shard * N, wpc = kPipeThreads / 32;
-    uint64_t ctas = 0, best_rounds = ~uint64_t(0);
-    for (int c = 1; c <= occ; ++c) {                  // fewest rounds of tiles, then fewest CTAs
-        const uint64_t w = uint64_t(sms) * c * wpc, rounds = (tiles + w - 1) / w;
-        if (rounds < best_rounds) {
-            best_rounds = rounds;
-            ctas = uint64_t(sms) * c;
-        }
-    }
-    ctas = std::min<uint64_t>(ctas, (tiles + wpc - 1) / wpc);
+    const uint64_t wpc = kPipeThreads / 32;
+    uint64_t ctas = persistent_grid(a.tiles_per_shard * N, wpc, sms, occ);
     if (keep_trace) ctas = std::min<uint64_t>(ctas, uint64_t(EQUARX_FLAVOUR_FIFO_BYTES) / (2 * kFifoEntryBytes) / wpc);
     if (keep_trace) {                                  // events that this flavour does not quantize stay zero
         e = cudaMemsetAsync(a.trace, 0, need - size_t(EQUARX_FLAVOUR_FIFO_BYTES), stream);

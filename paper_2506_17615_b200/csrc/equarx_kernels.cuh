@@ -494,8 +494,10 @@ struct Bf16GatherArgs {
 
 // ---------------------------------------------------------------- kernels
 // Ring step: FIRST = step 0 (quantize only), else dequantize-add-requantize.
-// Step 0 is never launched as a programmatic dependent: it reads tensors that an
-// earlier in-place all-gather on the same stream may still be writing.
+// Every launch may be a programmatic dependent of the kernel before it in the stream.  Step 0
+// reads tensors that the work before it may still be writing (an in-place all-gather, the
+// caller's producer), so it waits for that work before its first load; the later steps load
+// their bf16 shard, which nothing in this call writes before the all-gather, ahead of the wait.
 template <int LPB, bool FIRST, bool RECORDS>
 __global__ void __launch_bounds__(kThreads) rs_step_kernel(const __grid_constant__ StepArgs a) {
     const uint32_t r = blockIdx.y;
@@ -505,6 +507,7 @@ __global__ void __launch_bounds__(kThreads) rs_step_kernel(const __grid_constant
     const bool active = g < groups;
     const uint64_t pol = policy_keep();
 
+    if (FIRST) pdl_wait_prior_grid();
     Vec8 xw = {};
     if (active) xw = ld_stream_256(static_cast<const char*>(a.x[r]) + g * 32);
     pdl_launch_dependents();
@@ -701,17 +704,16 @@ __global__ void __launch_bounds__(kPipeThreads, EQX_PIPE_MINBLOCKS) pipelined_ke
 // bf16 inputs once and the bf16 outputs once (4 bytes per element of every rank).
 // The bf16 shard of the next rank of the chain is in flight while a step computes; DEPTH is the
 // number of such loads in flight per lane.
-#ifndef EQX_FUSED_MINBLOCKS
-#define EQX_FUSED_MINBLOCKS 18
-#endif
-#ifndef EQX_FUSED_DEPTH
-#define EQX_FUSED_DEPTH 1
-#endif
+// MINB = resident CTAs per SM the register allocation aims for.  Measured on B200: 18 (56 registers,
+// 36 warps per SM) is faster while the whole AllReduce moves little (below about 200 MB of input: the
+// launch is short and more warps fill the memory pipeline sooner), 16 (64 registers, 32 warps) is 2-5 %
+// faster above that.  The host picks per launch.
+constexpr int kFusedDepth = 1;
 
 // QUANT = false is the unquantized comparator in the same form: the message is the partial sum
 // rounded to bf16 and the receiving rank's add is rounded to bf16 again (the BF16 baseline's hop).
-template <int LPB, int DEPTH, bool QUANT>
-__global__ void __launch_bounds__(kPipeThreads, EQX_FUSED_MINBLOCKS) chain_fused_kernel(const __grid_constant__ PipeArgs a) {
+template <int LPB, int DEPTH, bool QUANT, int MINB>
+__global__ void __launch_bounds__(kPipeThreads, MINB) chain_fused_kernel(const __grid_constant__ PipeArgs a) {
     static_assert(DEPTH == 1 || DEPTH == 2, "one or two shards in flight");
     const uint32_t lane = threadIdx.x & 31u;
     const uint64_t warps = (uint64_t)gridDim.x * (kPipeThreads / 32);
@@ -1110,8 +1112,9 @@ __global__ void __launch_bounds__(kPipeThreads) flavour_fused_kernel(const __gri
 // ahead of the payload, microshards pipelined.  A rank's kernel is ONE persistent launch that runs
 // all N ring steps and the all-gather; a microshard is a 512-element tile, its message one
 // 544-byte record.  The sender stores the record straight into the RECEIVER's mailbox (plain
-// 16-byte stores: over NVLink when the mailbox lives on another GPU) and then releases a per-tile
-// flag word; the receiver's warp for that tile polls the flag with a BOUNDED wait.  Tiles advance
+// 16-byte stores: over NVLink when the mailbox lives on another GPU) and then, behind a system-scope
+// fence, sets a per-tile flag word; the receiver's warp for that tile polls the flag with a BOUNDED
+// wait (acquire loads).  Tiles advance
 // independently, so a tile's hop overlaps the transfers of all other tiles.  The last
 // reduce-scatter step stores the all-gather message of the rank's own shard into every rank's
 // mailbox (each peer is reachable at full bandwidth through the switch), and every rank
@@ -1130,6 +1133,7 @@ __global__ void __launch_bounds__(kPipeThreads) flavour_fused_kernel(const __gri
 // launch is cooperative) and exchange through the same mailboxes, which is how the whole ring runs
 // and is checked on a single GPU.
 constexpr int kRingThreads = 128;
+constexpr uint32_t kRingBatch = 4;      // tiles whose records share one system-scope fence
 constexpr uint32_t kRingOk = 0, kRingTimeout = 1;
 
 struct RingArgs {
@@ -1150,8 +1154,11 @@ __device__ __forceinline__ uint32_t ld_acquire_sys_u32(const uint32_t* p) {
     asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ void st_release_sys_u32(uint32_t* p, uint32_t v) {
-    asm volatile("st.release.sys.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+__device__ __forceinline__ void st_relaxed_sys_u32(uint32_t* p, uint32_t v) {
+    asm volatile("st.relaxed.sys.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void fence_acq_rel_sys() {
+    asm volatile("fence.acq_rel.sys;" ::: "memory");
 }
 // data written by another device (or another SM): strong loads, never served from a stale L1 line
 __device__ __forceinline__ uint4 ld_relaxed_sys_128(const void* p) {
@@ -1222,52 +1229,57 @@ __global__ void __launch_bounds__(kRingThreads) ring_rank_kernel(const __grid_co
     };
 
     // ---- reduce-scatter: step s sends shard (r - 1 - s) mod N
+    // A warp sends its tiles in batches of up to kRingBatch: the records of a batch are stored, ONE
+    // system-scope fence orders them, then the batch's flags are stored.  A fence across NVLink costs
+    // microseconds; the batch shares it.  A tile of step s waits only for tiles of step s - 1, so
+    // holding a flag back until its batch is complete cannot make a cycle of waits.
     for (uint32_t s = 0; s < N; ++s) {
         const uint32_t k = (r + 2 * N - 1 - s) % N;
-        for (uint64_t t = warp; t < T; t += warps) {
-            const bool active = t * 32 + lane < groups;
-            Vec8 xw = {};
-            if (active) xw = ld_coherent_256(x_rank + ((uint64_t)k * a.shard + (t * 32 + lane) * 16) * 2);   // in place is allowed
-            float v[16];
-            widen_bf16x16(xw, v);
-            if (s > 0) {                                              // the message received at this step
-                if (!ring_wait(flag_of(my_box, s - 1, t), a.epoch, a.timeout_ns, a.status, lane)) {
-                    fail(s, t);
-                    return;
+        const bool last = s + 1 == N;                                 // k == r: the shard is reduced
+        for (uint64_t t0 = warp; t0 < T; t0 += warps * kRingBatch) {
+            uint32_t sent = 0;
+            for (uint64_t t = t0; sent < kRingBatch && t < T; t += warps, ++sent) {
+                const bool active = t * 32 + lane < groups;
+                Vec8 xw = {};
+                if (active) xw = ld_coherent_256(x_rank + ((uint64_t)k * a.shard + (t * 32 + lane) * 16) * 2);   // in place is allowed
+                float v[16];
+                widen_bf16x16(xw, v);
+                if (s > 0) {                                          // the message received at this step
+                    if (!ring_wait(flag_of(my_box, s - 1, t), a.epoch, a.timeout_ns, a.status, lane)) {
+                        fail(s, t);
+                        return;
+                    }
+                    const char* rec = my_box + (uint64_t)(s - 1) * slot_bytes + t * kRecordBytes;
+                    uint4 c = make_uint4(0, 0, 0, 0);
+                    float sc = 0.0f;
+                    if (active) {
+                        c = ld_relaxed_sys_128(rec + kRecordHeader + lane * 16);
+                        sc = ld_relaxed_sys_f32(reinterpret_cast<const float*>(rec) + lane / LPB);
+                    }
+                    dequant_add_x16(c, sc, v);
                 }
-                const char* rec = my_box + (uint64_t)(s - 1) * slot_bytes + t * kRecordBytes;
-                uint4 c = make_uint4(0, 0, 0, 0);
-                float sc = 0.0f;
-                if (active) {
-                    c = ld_relaxed_sys_128(rec + kRecordHeader + lane * 16);
-                    sc = ld_relaxed_sys_f32(reinterpret_cast<const float*>(rec) + lane / LPB);
-                }
-                dequant_add_x16(c, sc, v);
-            }
-            uint4 codes;
-            float scale;
-            quantize_lane<LPB>(v, codes, scale, a.neg_zero);
-            float hdr = __shfl_sync(0xFFFFFFFFu, scale, (lane * LPB) & 31u);   // lanes 0..7: the metadata sector
-            if (lane >= 32u / LPB) hdr = 0.0f;
-            if (s + 1 < N) {
-                // to the right neighbour, as the message it receives at step s + 1
-                char* box = a.mailbox[right];
-                char* rec = box + (uint64_t)s * slot_bytes + t * kRecordBytes;
-                if (lane < 8) st_plain_f32(reinterpret_cast<float*>(rec) + lane, hdr);
-                if (active) st_plain_128(rec + kRecordHeader + lane * 16, codes);
-                __syncwarp();
-                if (lane == 0) st_release_sys_u32(flag_of(box, s, t), a.epoch);
-            } else {
-                // the reduced shard (k == r): its all-gather message goes to every rank
-                for (uint32_t q = 0; q < N; ++q) {
-                    char* box = a.mailbox[q];
-                    char* rec = box + (uint64_t)(N - 1 + k) * slot_bytes + t * kRecordBytes;
+                uint4 codes;
+                float scale;
+                quantize_lane<LPB>(v, codes, scale, a.neg_zero);
+                float hdr = __shfl_sync(0xFFFFFFFFu, scale, (lane * LPB) & 31u);   // lanes 0..7: the metadata sector
+                if (lane >= 32u / LPB) hdr = 0.0f;
+                // to the right neighbour, as the message it receives at step s + 1; the reduced shard's
+                // all-gather message goes to every rank
+                const uint32_t slot = last ? N - 1 + k : s;
+                for (uint32_t q = last ? 0 : right; q < (last ? N : right + 1); ++q) {
+                    char* rec = a.mailbox[q] + (uint64_t)slot * slot_bytes + t * kRecordBytes;
                     if (lane < 8) st_plain_f32(reinterpret_cast<float*>(rec) + lane, hdr);
                     if (active) st_plain_128(rec + kRecordHeader + lane * 16, codes);
                 }
-                __syncwarp();
-                if (lane == 0)
-                    for (uint32_t q = 0; q < N; ++q) st_release_sys_u32(flag_of(a.mailbox[q], N - 1 + k, t), a.epoch);
+            }
+            __syncwarp();                                             // every lane's stores happen before lane 0's fence
+            if (lane == 0) {
+                fence_acq_rel_sys();
+                const uint32_t slot = last ? N - 1 + k : s;
+                uint64_t t = t0;
+                for (uint32_t i = 0; i < sent; ++i, t += warps)
+                    for (uint32_t q = last ? 0 : right; q < (last ? N : right + 1); ++q)
+                        st_relaxed_sys_u32(flag_of(a.mailbox[q], slot, t), a.epoch);
             }
         }
     }
