@@ -51,7 +51,7 @@ L2_BYTES = 126_000_000
 # from DRAM.
 NCU_TRAFFIC = {
     "chain_fused_kernel": {"bytes_per_element": 4.0, "profile": "profiles/chain_fused_kernel_c2_c3.md"},
-    "rs_step_hop_small": {"bytes_per_element": 3.017, "profile": "profiles/rs_step_kernel_c2_full.md"},
+    "rs_step_hop_small": {"bytes_per_element": 3.06, "profile": "profiles/rs_step_kernel_c2_full.md"},
     "rs_step_hop_large": {"bytes_per_element": 3.95, "profile": "profiles/rs_step_kernel_c2_full.md"},
 }
 HOP_MESSAGES_STAY_IN_L2_BYTES = 20_000_000

@@ -6,6 +6,8 @@
 
 #include <algorithm>
 #include <atomic>
+#include <mutex>
+#include <vector>
 #include <cstdlib>
 #include <cstring>
 
@@ -114,6 +116,43 @@ int launch_gather(int block, const GatherArgs& a, cudaStream_t stream, bool depe
         case 256: return launch(ag_dequant_kernel<16, RECORDS>, grid, a, stream, dependent);
         default: return launch(ag_dequant_kernel<32, RECORDS>, grid, a, stream, dependent);
     }
+}
+
+// Launch geometry of a persistent kernel depends on the device (SM count) and on the kernel's
+// occupancy; both are constant for the life of the process, so they are looked up once per
+// (device, kernel) and remembered: the queries cost about as much as the launch itself.
+struct Residency {
+    int sms = 0, occ = 0, coop = 0;
+};
+
+cudaError_t residency_of(const void* kernel, int threads, Residency& out) {
+    struct Entry {
+        int dev;
+        const void* kernel;
+        Residency r;
+    };
+    static std::mutex mu;
+    static std::vector<Entry> seen;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        for (const Entry& en : seen)
+            if (en.dev == dev && en.kernel == kernel) {
+                out = en.r;
+                return cudaSuccess;
+            }
+    }
+    Residency r;
+    e = cudaDeviceGetAttribute(&r.sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&r.coop, cudaDevAttrCooperativeLaunch, dev);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&r.occ, kernel, threads, 0);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(mu);
+    seen.push_back(Entry{dev, kernel, r});
+    out = r;
+    return cudaSuccess;
 }
 
 // Persistent grid of the single-launch kernels: a whole number of CTAs per SM (measured: a grid that
@@ -406,10 +445,9 @@ int launch_pipelined(const void* const* in_bf16, void* const* out_bf16, int nran
 #undef EQX_FUSED
 #undef EQX_PICK
     // persistent grid: a whole number of CTAs per SM
-    int dev = 0, sms = 0, occ = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kPipeThreads, 0);
+    Residency res;
+    cudaError_t e = residency_of(kernel, kPipeThreads, res);
+    const int sms = res.sms, occ = res.occ;
     if (e != cudaSuccess || sms < 1 || occ < 1) {
         g_last_cuda_error = int(e);
         (void)cudaGetLastError();
@@ -549,10 +587,9 @@ int equarx_allreduce_sim_flavour(const void* const* in_bf16, void* const* out_bf
         case 256: kernel = keep_trace ? flavour_kernel_for<16>(flavour) : flavour_fused_kernel_for<16>(flavour); break;
         default: kernel = keep_trace ? flavour_kernel_for<32>(flavour) : flavour_fused_kernel_for<32>(flavour); break;
     }
-    int dev = 0, sms = 0, occ = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kPipeThreads, 0);
+    Residency res;
+    cudaError_t e = residency_of(kernel, kPipeThreads, res);
+    const int sms = res.sms, occ = res.occ;
     if (e != cudaSuccess || sms < 1 || occ < 1) {
         g_last_cuda_error = int(e);
         (void)cudaGetLastError();
@@ -649,11 +686,9 @@ int equarx_ring_allreduce(const void* const* in_bf16, void* const* out_bf16, int
         (void)cudaGetLastError();
         return EQUARX_ERR_CUDA;
     };
-    int dev = 0, sms = 0, occ = 0, coop = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
-    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kRingThreads, 0);
+    Residency res;
+    cudaError_t e = residency_of(kernel, kRingThreads, res);
+    const int sms = res.sms, occ = res.occ, coop = res.coop;
     if (e != cudaSuccess) return failed(e);
     if (sms < 1 || occ < 1 || !coop) return failed(cudaErrorCooperativeLaunchTooLarge);
     // every hosted rank gets the same number of CTAs and all of them must be resident at once

@@ -21,7 +21,10 @@
 
 namespace equarx {
 
-constexpr int kThreads = 256;        // threads per CTA
+#ifndef EQX_STEP_THREADS
+#define EQX_STEP_THREADS 256
+#endif
+constexpr int kThreads = EQX_STEP_THREADS;        // threads per CTA of the per-step kernels
 constexpr int kLaneElems = 16;       // elements per lane
 constexpr int kMaxRanks = 64;
 
