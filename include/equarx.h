@@ -366,8 +366,9 @@ int equarx_allreduce_sim_static(const void *const *in_bf16, void *const *out_bf1
  *                 {EQUARX_RING_TIMEOUT, rank, step, tile} in `status` (first failure
  *                 only) and leave; the kernel always terminates, never traps.  step is
  *                 the ring step, or nranks + shard for an all-gather message.
- *   status      : DEVICE memory, 4 x uint32, 16-byte aligned, zeroed by the caller;
- *                 read it after synchronising: code 0 means every message arrived.
+ *   status      : DEVICE memory, 4 x uint32, 16-byte aligned; cleared by this call on
+ *                 `stream` ahead of the kernel; read it after synchronising: code 0
+ *                 means every message arrived.
  * Returns EQUARX_ERR_CUDA if the cooperative launch is refused (for example more hosted
  * ranks than CTAs that fit on the device).
  * Not exercised on more than one GPU; the ranks_here = nranks form is what the tests run.

@@ -171,7 +171,7 @@ def ring_mailbox_bytes(nranks, count, block):
 def ring_allreduce(in_bf16, out_bf16, rank_first, ranks_here, nranks, count, block, mailboxes, epoch, timeout_ns,
                    status, stream=0):
     """equarx_ring_allreduce: the ranks rank_first .. rank_first+ranks_here-1 of the ring on the current
-    device; `mailboxes` lists every rank's mailbox, `status` is 4 zeroed uint32 words on the device."""
+    device; `mailboxes` lists every rank's mailbox, `status` is 4 uint32 words on the device (cleared by the call)."""
     _check(lib.equarx_ring_allreduce(_table(in_bf16), _table(out_bf16), rank_first, ranks_here, nranks, count, block,
                                      _table(mailboxes), epoch, timeout_ns, _ptr(status), _ptr(stream)),
            "equarx_ring_allreduce")

@@ -1202,6 +1202,7 @@ __device__ __forceinline__ bool ring_wait(const uint32_t* flag, uint32_t epoch, 
         }
     }
     ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+    __syncwarp();                    // orders the other lanes' record loads after lane 0's acquire
     return ok != 0;
 }
 

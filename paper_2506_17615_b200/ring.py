@@ -136,7 +136,6 @@ class LocalRing:
         """ins, outs: N bf16 device tensors.  Asynchronous; check() synchronises and raises on a time-out."""
         lay = self.layout
         self.epoch += 1
-        self.status.zero_()
         self._b.ring_allreduce(ins, outs, 0, lay.nranks, lay.nranks, lay.count, lay.block, self.mailboxes,
                                self.epoch, timeout_ns, self.status, stream)
 
@@ -226,7 +225,6 @@ class PeerRing:
         """x, out: this rank's bf16 tensors (count elements).  All ranks call it the same number of times."""
         lay = self.layout
         self.epoch += 1
-        self.status.zero_()
         self._launch([x], [out], self.rank, 1, lay.nranks, lay.count, lay.block, self.mailboxes, self.epoch,
                      timeout_ns, self.status, stream)
 
