@@ -548,7 +548,7 @@ def main():
                 "hop_traffic_bytes_per_launch": hop["bytes_per_element"] * count,
                 "hop_traffic_source": f"ncu, {hop['profile']}, scaled by elements"}
 
-    flavours, bf16_sim, ratios, ring_local = {}, None, None, None
+    flavours, bf16_sim, ratios, ring_local, graph_replay = {}, None, None, None, None
     if not args.no_extras:
         # ---- the other flavours (semi-loop ring, stage selection, FP8), same workload, single launch
         wbf = eq.allreduce_sim_flavour_workspace_bytes(N, count, block, 7 if N % 2 == 0 else 6, False)
@@ -583,6 +583,28 @@ def main():
                                      "once; the all-gather message of every shard written to and read from N mailboxes",
                       "frac": ring_bytes / (ms_r * 1e-3) / 1e9 / peak}
         del lring
+
+        # ---- both schedules recorded once per input set by stream capture and replayed as CUDA graphs
+        # (removes the host-call and launch overhead that bounds small messages)
+        graph_replay = {}
+        for gname, fn in (("single_launch", step_fused), ("by_steps", step_by_steps)):
+            graphs = []
+            side = torch.cuda.Stream(dev)
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                for s_ in range(sets):
+                    g_ = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g_, stream=side):
+                        capture_stream = torch.cuda.current_stream().cuda_stream
+                        if gname == "single_launch":
+                            eq.allreduce_sim_pipelined(ins[s_], outs[s_], N, count, block, wsp, wbp, False, capture_stream)
+                        else:
+                            eq.allreduce_sim(ins[s_], outs[s_], N, count, block, ws, wb, False, capture_stream)
+                    graphs.append(g_)
+            torch.cuda.current_stream().wait_stream(side)
+            ms_g, _ = timed(lambda i: graphs[i % sets].replay(), args.steps, min_seconds=0.2)
+            graph_replay[gname] = {"ms_per_step": ms_g, "value": aggregate_value(in_bytes, ms_g, world), "unit": UNIT}
+            del graphs
 
         # ---- unquantized comparator on the same GPU, same inputs, one launch per ring step
         wb16 = eq.allreduce_sim_bf16_workspace_bytes(N, count)
@@ -653,7 +675,7 @@ def main():
             "e2e": e2e, "gpu_launches": args.steps, "clocks": clocks,
             "roofline": roofline,
             "schedule": "chain-fused single launch (equarx_allreduce_sim_pipelined, keep_trace=0)",
-            "by_steps": by_steps, "ring_on_one_gpu": ring_local, "flavours": flavours, "bf16_sim": bf16_sim,
+            "by_steps": by_steps, "ring_on_one_gpu": ring_local, "graph_replay": graph_replay, "flavours": flavours, "bf16_sim": bf16_sim,
             "speedup_vs_bf16": ratios, "input_checksum": checksum,
             "pdl_between_step_launches": os.environ.get("EQUARX_PDL", "1") != "0",
         }

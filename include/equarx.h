@@ -14,7 +14,12 @@
  *     enqueued.  For tests, EQUARX_INJECT_LAUNCH_ERROR=<code> in the environment makes
  *     every launch report that code without launching anything.
  *   - Work is enqueued on `stream` and the call returns without
- *     synchronising.  Device buffers must stay valid until the stream has
+ *     synchronising.  The per-step calls, equarx_allreduce_sim(_range),
+ *     equarx_allreduce_sim_pipelined, equarx_allreduce_sim_flavour and
+ *     equarx_allreduce_sim_bf16 only enqueue kernel launches (and one memset for a
+ *     flavour trace), so they can be recorded by stream capture and replayed as a
+ *     CUDA graph; for messages below a few MB per rank, where launch and call
+ *     overhead dominate, a replay takes about half the time of the direct calls.  Device buffers must stay valid until the stream has
  *     reached the work.  The library allocates and frees nothing: the caller
  *     owns every buffer, including the workspace.
  *   - Pointer tables (`in_bf16`, `out_bf16`) are HOST arrays of DEVICE

@@ -810,6 +810,8 @@ __global__ void __launch_bounds__(kPipeThreads, MINB) chain_fused_kernel(const _
 // carries a 512-element tile along its adder chain(s); every message goes through the
 // warp's two-entry staging FIFO and is read back by the neighbouring lane.  A message
 // is a 544-byte quantized record or, for an unquantized stage, 1024 bytes of bf16.
+// flavour_kernel is the form used when a trace is kept (every quantized message is also
+// written to the trace); flavour_fused_kernel further down keeps the messages in registers.
 constexpr int kFifoEntryBytes = 1024;
 
 struct FlavourArgs {

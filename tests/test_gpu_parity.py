@@ -479,6 +479,40 @@ def test_runs_on_the_stream_it_is_given(gu):
     gu.assert_same_words(out, exp, "side stream")
 
 
+def test_schedules_can_be_recorded_in_a_cuda_graph(gu):
+    """The simulation calls only enqueue launches on the given stream (no synchronisation, no allocation),
+    so stream capture records them; replaying the graph on new data gives the oracle's bits.  Small
+    messages are bound by launch and host-call overhead, which a graph replay removes."""
+    n, block = 4, 256
+    count = n * block * 24
+    x = torch.zeros((n, count), dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros_like(x)
+    ins, outs = [x[r] for r in range(n)], [out[r] for r in range(n)]
+    wb = eq.allreduce_sim_workspace_bytes(n, count, block, False)
+    ws = torch.empty(wb, dtype=torch.uint8, device="cuda")
+    wbf = eq.allreduce_sim_flavour_workspace_bytes(n, count, block, 7, False)
+    calls = {"launch per step": lambda s: eq.allreduce_sim(ins, outs, n, count, block, ws, wb, False, s),
+             "single launch": lambda s: eq.allreduce_sim_pipelined(ins, outs, n, count, block, ws, wb, False, s),
+             "semi-loop flavour": lambda s: eq.allreduce_sim_flavour(ins, outs, n, count, block, 7, ws, wbf, False, s)}
+    for name, call in calls.items():
+        call(gu.stream_handle())                       # first use outside capture: loads the kernels
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            call(torch.cuda.current_stream().cuda_stream)
+        for seed in (61, 62):
+            src = wl.make_inputs(wl.Workload("t", n, count, block, "normal", seed=seed))
+            x.copy_(src)
+            out.zero_()
+            graph.replay()
+            torch.cuda.synchronize()
+            if name == "semi-loop flavour":
+                exp = oracle.allreduce_variant(wl.as_u16(src), block, True, True, True)["out"]
+            else:
+                exp = oracle.allreduce(wl.as_u16(src), block)["out"]
+            gu.assert_same_words(out, exp, f"{name}, graph replay, seed {seed}")
+
+
 def test_launch_errors_are_reported_not_raised_on_the_gpu(gu, monkeypatch):
     """A failing launch (injected on the host: no kernel runs, the GPU is not touched) comes back
     as EQUARX_ERR_CUDA with the CUDA error code available, from every kind of entry point, and
