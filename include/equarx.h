@@ -3,7 +3,8 @@
  * of EQuARX (arXiv 2506.17615): dynamic block-wise int8 quantization and the
  * dequantize / fp32-accumulate / requantize work that runs beside the steps
  * of a ring AllReduce, simulated on ONE GPU over N logical ranks whose bf16
- * buffers all live in that GPU's memory.
+ * buffers all live in that GPU's memory.  equarx_ring_allreduce, at the end,
+ * is the same arithmetic as a ring with one rank per device.
  *
  * Conventions for every function
  *   - extern "C"; returns an EQUARX_* status; never throws, aborts or exits.
@@ -19,9 +20,10 @@
  *     equarx_allreduce_sim_bf16 only enqueue kernel launches (and one memset for a
  *     flavour trace), so they can be recorded by stream capture and replayed as a
  *     CUDA graph; for messages below a few MB per rank, where launch and call
- *     overhead dominate, a replay takes about half the time of the direct calls.  Device buffers must stay valid until the stream has
- *     reached the work.  The library allocates and frees nothing: the caller
- *     owns every buffer, including the workspace.
+ *     overhead dominate, a replay takes about half the time of the direct calls.
+ *   - Device buffers must stay valid until the stream has reached the work.
+ *     The library allocates and frees nothing: the caller owns every buffer,
+ *     including the workspace.
  *   - Pointer tables (`in_bf16`, `out_bf16`) are HOST arrays of DEVICE
  *     pointers; they are copied into kernel parameters during the call and
  *     may be freed as soon as it returns.  All other pointers are DEVICE

@@ -1123,7 +1123,7 @@ __global__ void __launch_bounds__(kPipeThreads) flavour_fused_kernel(const __gri
 // independently, so a tile's hop overlaps the transfers of all other tiles.  The last
 // reduce-scatter step stores the all-gather message of the rank's own shard into every rank's
 // mailbox (each peer is reachable at full bandwidth through the switch), and every rank
-// dequantizes what it received.  No bulk-tensor copy and no multicast of any kind is used.
+// dequantizes what it received.  Only plain loads and stores touch peer memory: no bulk-tensor copy, no one-to-many load.
 //
 // Mailbox of a rank (device memory, zeroed once before its first use):
 //   slots 0..N-2   : the message received at ring step s = slot + 1 (tiles_per_shard records)
