@@ -85,3 +85,29 @@ def test_sweep_summary_from_a_results_file(tmp_path):
     text = sweep.summarize(str(path))
     assert "| 8 | 256 | 1 MB | 1000 (0.400)" in text and "| 8 | 256 | 64 MB | 1000 (0.960)" in text
     assert "All 1 points with at least 64 MB per rank: single launch 0.960 - 0.960" in text
+
+
+@pytest.mark.gpu
+def test_bench_line_on_the_gpu_is_consistent():
+    """One short run on the smallest config: the line carries the contract's keys, each roofline fraction
+    is its bytes over its time over its peak, the parity verdict is bit-exact, e2e moved the bytes it names."""
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--workload", "C1", "--steps", "5",
+                          "--min-seconds", "0.02"], capture_output=True, text=True, timeout=900)
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
+                "vs_baseline", "dtype", "data", "config", "e2e", "gpu_launches", "clocks", "roofline", "cpu_baseline"):
+        assert key in line, key
+    n, count, block = 4, 65536, 256
+    assert line["config"]["workload"].startswith("C1") and line["gpu_launches"] == 5
+    r = line["roofline"]
+    assert r["bytes_per_launch"] == 4 * count * n and r["kernel"] == "chain_fused_kernel"
+    assert r["achieved"] == pytest.approx(r["bytes_per_launch"] / (line["ms_per_step"] * 1e-3) / 1e9, rel=1e-9)
+    assert r["frac"] == pytest.approx(r["achieved"] / r["peak"], rel=1e-9)
+    assert line["value"] == pytest.approx(2 * count * n / (line["ms_per_step"] * 1e-3) / 1e9, rel=1e-9)
+    b = line["by_steps"]["roofline"]
+    assert b["bytes_per_launch"] == count * n * (6 + 8 / block)
+    assert b["frac"] == pytest.approx(b["bytes_per_launch"] / (line["by_steps"]["ms_per_step"] * 1e-3) / 1e9 / b["peak"], rel=1e-9)
+    assert line["parity"]["verdict"] == "bit-exact" and line["parity"]["checked_words"] == n * count
+    assert line["e2e"]["h2d_bytes_per_step"] == 2 * count * n == line["e2e"]["d2h_bytes_per_step"]
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] == 1

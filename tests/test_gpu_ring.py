@@ -156,3 +156,21 @@ def test_mailbox_handles_map_the_same_memory_in_another_process():
         assert int(err) == 0 and (host == 0x3C).all()
     finally:
         mem.free(ptr)
+
+
+def test_bench_ring_mode_with_a_single_rank():
+    """bench.py --ring runs PeerRing end to end (mailbox allocation, IPC export, the process group, the
+    launch with ranks_here = 1, status read-back, close); with one process the ring has one rank."""
+    import json
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    env["MASTER_PORT"] = str(29600 + os.getpid() % 300)
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--ring", "--workload", "C1", "--steps", "3",
+                          "--min-seconds", "0"], env=env, capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    assert line["failure"] is None and line["value"] > 0 and line["config"]["nranks"] == 1
+    assert "ranks_here=1" in line["schedule"]
