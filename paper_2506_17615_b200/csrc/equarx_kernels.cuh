@@ -501,8 +501,10 @@ struct Bf16GatherArgs {
 // reads tensors that the work before it may still be writing (an in-place all-gather, the
 // caller's producer), so it waits for that work before its first load; the later steps load
 // their bf16 shard, which nothing in this call writes before the all-gather, ahead of the wait.
+// 8 CTAs of 256 threads per SM (32 registers, full occupancy): 2-3 % faster than the 34 registers and
+// 7 CTAs the compiler picks on its own (B200, 16 MB and 88 MB per rank).
 template <int LPB, bool FIRST, bool RECORDS>
-__global__ void __launch_bounds__(kThreads) rs_step_kernel(const __grid_constant__ StepArgs a) {
+__global__ void __launch_bounds__(kThreads, 2048 / kThreads) rs_step_kernel(const __grid_constant__ StepArgs a) {
     const uint32_t r = blockIdx.y;
     const uint32_t lane = threadIdx.x & 31u;
     const uint64_t g = (uint64_t)blockIdx.x * kThreads + threadIdx.x;   // 16-element group
