@@ -22,9 +22,20 @@ def gu():
     return gpu_util
 
 
+def guard_mailboxes(gu, ring):
+    """Replace the ring's mailboxes by zeroed buffers with canary bands on both sides (once per ring)."""
+    if getattr(ring, "_guards", None) is None:
+        ring._guards = [gu.Guarded(ring.layout.mailbox_bytes) for _ in range(ring.layout.nranks)]
+        for g in ring._guards:
+            g.u8.zero_()
+        ring.mailboxes = [g.u8 for g in ring._guards]
+    return ring._guards
+
+
 def run_and_compare(gu, ring, x, in_place=False):
     n, count = x.shape
     block = ring.layout.block
+    guards = guard_mailboxes(gu, ring)
     res = oracle.allreduce(wl.as_u16(x), block, trace=True)
     xd = x.cuda()
     if in_place:
@@ -37,7 +48,7 @@ def run_and_compare(gu, ring, x, in_place=False):
         outs = [gu.Guarded(2 * count) for _ in range(n)]
     ring.allreduce(ins, outs, stream=gu.stream_handle())
     ring.check()
-    for o in outs:
+    for o in outs + guards:
         o.check()
     out = torch.stack([o.view(torch.bfloat16) for o in outs])
     gu.assert_same_words(out, res["out"], "ring outputs")
