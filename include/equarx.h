@@ -370,18 +370,18 @@ int equarx_allreduce_sim_static(const void *const *in_bf16, void *const *out_bf1
  *                 Calls that share mailboxes must be ordered on each rank's stream.
  *   timeout_ns  : longest wait for one message; 0 selects 1 second.  A wait that runs
  *                 out, or that sees another warp's failure, makes the warp record
- *                 {EQUARX_RING_TIMEOUT, rank, step, tile} in `status` (first failure
+ *                 {epoch, rank, step, tile} in `status` (first failure of the call
  *                 only) and leave; the kernel always terminates, never traps.  step is
  *                 the ring step, or nranks + shard for an all-gather message.
- *   status      : DEVICE memory, 4 x uint32, 16-byte aligned; cleared by this call on
- *                 `stream` ahead of the kernel; read it after synchronising: code 0
- *                 means every message arrived.
+ *   status      : DEVICE memory, 4 x uint32, 16-byte aligned, zeroed ONCE by the caller
+ *                 before its first use (like the mailboxes); nothing clears it between
+ *                 calls.  Read it after synchronising: status[0] equal to the call's
+ *                 epoch means that call timed out, any other value that every
+ *                 message of the call arrived.
  * Returns EQUARX_ERR_CUDA if the cooperative launch is refused (for example more hosted
  * ranks than CTAs that fit on the device).
  * Not exercised on more than one GPU; the ranks_here = nranks form is what the tests run.
  */
-#define EQUARX_RING_OK 0u
-#define EQUARX_RING_TIMEOUT 1u
 size_t equarx_ring_mailbox_bytes(int nranks, size_t count, int block);
 int equarx_ring_allreduce(const void *const *in_bf16, void *const *out_bf16,
                           int rank_first, int ranks_here, int nranks, size_t count, int block,

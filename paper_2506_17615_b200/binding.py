@@ -161,9 +161,6 @@ def allreduce_sim_host(host_in, host_out, nranks, count, block, staging, staging
            "equarx_allreduce_sim_host")
 
 
-RING_OK, RING_TIMEOUT = 0, 1
-
-
 def ring_mailbox_bytes(nranks, count, block):
     return lib.equarx_ring_mailbox_bytes(nranks, count, block)
 
@@ -171,7 +168,7 @@ def ring_mailbox_bytes(nranks, count, block):
 def ring_allreduce(in_bf16, out_bf16, rank_first, ranks_here, nranks, count, block, mailboxes, epoch, timeout_ns,
                    status, stream=0):
     """equarx_ring_allreduce: the ranks rank_first .. rank_first+ranks_here-1 of the ring on the current
-    device; `mailboxes` lists every rank's mailbox, `status` is 4 uint32 words on the device (cleared by the call)."""
+    device; `mailboxes` lists every rank's mailbox, `status` is 4 uint32 words on the device, zeroed once; status[0] == epoch after a call means it timed out."""
     _check(lib.equarx_ring_allreduce(_table(in_bf16), _table(out_bf16), rank_first, ranks_here, nranks, count, block,
                                      _table(mailboxes), epoch, timeout_ns, _ptr(status), _ptr(stream)),
            "equarx_ring_allreduce")

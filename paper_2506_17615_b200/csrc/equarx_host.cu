@@ -700,7 +700,6 @@ int equarx_ring_allreduce(const void* const* in_bf16, void* const* out_bf16, int
     a.ctas_per_rank = uint32_t(per_rank);
     void* params[1] = {&a};
     e = injected_launch_error();
-    if (e == cudaSuccess) e = cudaMemsetAsync(status, 0, 4 * sizeof(uint32_t), stream);   // "no failure so far"
     if (e == cudaSuccess)
         e = cudaLaunchCooperativeKernel(kernel, dim3(unsigned(per_rank * uint64_t(ranks_here))), dim3(kRingThreads),
                                         params, 0, stream);

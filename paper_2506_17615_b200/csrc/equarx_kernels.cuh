@@ -1139,15 +1139,20 @@ __global__ void __launch_bounds__(kPipeThreads) flavour_fused_kernel(const __gri
 // A launch can host several consecutive ranks (ranks_here > 1): their CTAs are co-resident (the
 // launch is cooperative) and exchange through the same mailboxes, which is how the whole ring runs
 // and is checked on a single GPU.
-constexpr int kRingThreads = 128;
-constexpr uint32_t kRingBatch = 4;      // tiles whose records share one system-scope fence
-constexpr uint32_t kRingOk = 0, kRingTimeout = 1;
+#ifndef EQX_RING_THREADS
+#define EQX_RING_THREADS 128
+#endif
+#ifndef EQX_RING_BATCH
+#define EQX_RING_BATCH 8
+#endif
+constexpr int kRingThreads = EQX_RING_THREADS;
+constexpr uint32_t kRingBatch = EQX_RING_BATCH;      // tiles whose records share one system-scope fence
 
 struct RingArgs {
     const void* in[kMaxRanks];       // input tensor of hosted rank rank_first + i
     void* out[kMaxRanks];            // output tensor of hosted rank rank_first + i
     char* mailbox[kMaxRanks];        // mailbox of EVERY rank of the ring, as addressable from this device
-    uint32_t* status;                // {code, rank, step, tile}: first failure of this launch, else untouched
+    uint32_t* status;                // {epoch of the failed call, rank, step, tile}: first failure of this launch, else untouched
     uint64_t shard;
     uint64_t tiles_per_shard;
     uint64_t timeout_ns;             // longest wait for one message
@@ -1197,7 +1202,7 @@ __device__ __forceinline__ bool ring_wait(const uint32_t* flag, uint32_t epoch, 
             for (uint32_t spins = 1;; ++spins) {
                 if (ld_acquire_sys_u32(flag) == epoch) break;
                 if ((spins & 15u) == 0 &&
-                    (global_timer_ns() - t0 > timeout_ns || *reinterpret_cast<const volatile uint32_t*>(status) != 0)) {
+                    (global_timer_ns() - t0 > timeout_ns || *reinterpret_cast<const volatile uint32_t*>(status) == epoch)) {
                     ok = 0;
                     break;
                 }
@@ -1228,11 +1233,15 @@ __global__ void __launch_bounds__(kRingThreads) ring_rank_kernel(const __grid_co
     auto flag_of = [&](char* box, uint32_t slot, uint64_t t) {
         return reinterpret_cast<uint32_t*>(box + flags_at) + (uint64_t)slot * T + t;
     };
-    auto fail = [&](uint32_t step, uint64_t t) {                      // first failure wins; then this warp leaves
-        if (lane == 0 && atomicCAS(a.status, kRingOk, kRingTimeout) == kRingOk) {
-            a.status[1] = r;
-            a.status[2] = step;
-            a.status[3] = (uint32_t)t;
+    // a failing call stamps the status with its own epoch (first failure wins); then this warp leaves
+    auto fail = [&](uint32_t step, uint64_t t) {
+        if (lane == 0) {
+            const uint32_t seen = *reinterpret_cast<volatile uint32_t*>(a.status);
+            if (seen != a.epoch && atomicCAS(a.status, seen, a.epoch) == seen) {
+                a.status[1] = r;
+                a.status[2] = step;
+                a.status[3] = (uint32_t)t;
+            }
         }
     };
 

@@ -110,9 +110,10 @@ class RingLayout:
         return scales, codes
 
 
-def _raise_on_status(words, nranks):
-    code, rank, step, tile = (int(w) for w in words)
-    if code != 0:
+def _raise_on_status(words, nranks, epoch):
+    """A failed call stamps the status with its epoch; any other first word means the call completed."""
+    code, rank, step, tile = (int(w) & 0xFFFFFFFF for w in words)
+    if epoch > 0 and code == epoch:
         raise RingTimeout(rank, step, tile, nranks)
 
 
@@ -142,7 +143,7 @@ class LocalRing:
     def check(self):
         import torch
         torch.cuda.synchronize(self.device)
-        _raise_on_status(self.status.cpu().tolist(), self.layout.nranks)
+        _raise_on_status(self.status.cpu().tolist(), self.layout.nranks, self.epoch)
 
     def trace(self):
         return self.layout.trace([m.cpu().numpy() for m in self.mailboxes])
@@ -236,7 +237,7 @@ class PeerRing:
             words = self.status.cpu().tolist()
         else:
             words = list(self.status)
-        _raise_on_status(words, self.layout.nranks)
+        _raise_on_status(words, self.layout.nranks, self.epoch)
 
     def close(self):
         """Between calls only: no kernel of any rank may still be using the mailboxes."""

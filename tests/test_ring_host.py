@@ -103,12 +103,13 @@ def test_ring_entry_rejects_bad_arguments_before_any_cuda_call():
 
 
 def test_status_words_become_an_exception():
-    _raise_on_status([0, 0, 0, 0], 4)
+    _raise_on_status([0, 0, 0, 0], 4, epoch=5)
+    _raise_on_status([4, 2, 3, 17], 4, epoch=5)              # an earlier call failed, this one did not
     with pytest.raises(RingTimeout) as e:
-        _raise_on_status([1, 2, 3, 17], 4)
+        _raise_on_status([5, 2, 3, 17], 4, epoch=5)
     assert (e.value.rank, e.value.step, e.value.tile) == (2, 3, 17) and "ring step 3" in str(e.value)
     with pytest.raises(RingTimeout) as e:
-        _raise_on_status([1, 0, 4 + 2, 5], 4)
+        _raise_on_status([9, 0, 4 + 2, 5], 4, epoch=9)
     assert "all-gather message of shard 2" in str(e.value)
 
 
@@ -147,9 +148,8 @@ def _peer_worker(rank, world, port, q, fail_rank):
     def launch(ins, outs, rank_first, ranks_here, nranks, count, block, mailboxes, epoch, timeout_ns, st, stream):
         calls.append(dict(rank_first=rank_first, ranks_here=ranks_here, nranks=nranks, mailboxes=list(mailboxes),
                           epoch=epoch, timeout_ns=timeout_ns))
-        st[:] = [0, 0, 0, 0]                               # the library clears the status ahead of the kernel
         if rank == fail_rank and epoch == 2:               # the kernel would have written this after a time-out
-            st[:] = [1, rank, 1, 0]
+            st[:] = [epoch, rank, 1, 0]
 
     ring = PeerRing(2 * 256 * 3, 256, memory=FakeMemory(rank, log), launch=launch, status=status)
     ring.allreduce("x", "out")
