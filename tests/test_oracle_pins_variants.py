@@ -249,3 +249,29 @@ def test_adder_tree_exact_rational(payload, kind, semi, qr, qa, nranks, block, b
         assert int(res["scales"][k, j, b].view(np.uint32)) == f32_word(scale), (k, b, j)
         got = [_fp8_or_int(c, payload) for c in res["codes"][k, j, b * block:(b + 1) * block]]
         assert got == [float(v) for v in vals], (k, b, j)
+
+
+# ---------------------------------------------------------------- randomized shapes (hypothesis)
+from hypothesis import HealthCheck, given, settings, strategies as st   # noqa: E402
+
+
+@settings(max_examples=60, deadline=None, suppress_health_check=[HealthCheck.too_slow])
+@given(half=st.integers(1, 4), block=st.integers(1, 6), bps=st.integers(1, 2),
+       flavour=st.integers(0, 7), payload=st.sampled_from(["int8", "e4m3", "e5m2"]),
+       kind=st.sampled_from(["normal", "wide", "halves", "tiny"]), seed=st.integers(0, 2 ** 31 - 1))
+def test_random_shapes_against_the_exact_rational_tree(half, block, bps, flavour, payload, kind, seed):
+    """Any even rank count up to 8, any block length, every flavour and payload: the oracle equals the
+    rational evaluation of the adder chain / tree bit for bit."""
+    from test_oracle_pins_chain import rand_bf16
+    from exact_fp import f32_word, tree_allreduce
+    semi, qr, qa = bool(flavour & 1), bool(flavour & 2), bool(flavour & 4)
+    nranks = 2 * half
+    x = rand_bf16(np.random.default_rng(seed), (nranks, nranks * block * bps), kind)
+    res = oracle.allreduce_variant(x, block, semi, qr, qa, trace=True, payload=payload)
+    out, events = tree_allreduce([[int(w) for w in row] for row in x], block, semi, qr, qa, payload)
+    for r in range(nranks):
+        assert [0 if int(w) == 0x8000 else int(w) for w in res["out"][r]] == out
+    for (k, b, j), (scale, vals) in events.items():
+        assert int(res["scales"][k, j, b].view(np.uint32)) == f32_word(scale)
+        got = [_fp8_or_int(c, payload) for c in res["codes"][k, j, b * block:(b + 1) * block]]
+        assert got == [float(v) for v in vals]
