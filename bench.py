@@ -50,7 +50,11 @@ L2_BYTES = 126_000_000
 # fit the part of L2 that keeps them, about 20 MB; above that it is written back and read again
 # from DRAM.
 NCU_TRAFFIC = {
-    "chain_fused_kernel": {"bytes_per_element": 4.0, "profile": "profiles/chain_fused_kernel_c2_c3.md"},
+    "chain_fused_kernel": {"bytes_per_element": 4.0, "profile": "profiles/chain_fused_kernel_c2_c3.md",
+                           # read + written while the kernel runs, as captured (the rest of the outputs is still
+                           # dirty in L2 when the kernel ends and is written back during the next launch)
+                           "captured": {"C2_gemma3_12b_prefill2048": 125.85e6 + 68.15e6,
+                                        "C3_gemma3_27b_prefill8192": 704.66e6 + 651.57e6}},
     "rs_step_hop_small": {"bytes_per_element": 3.06, "profile": "profiles/rs_step_kernel_c2_full.md"},
     "rs_step_hop_large": {"bytes_per_element": 3.95, "profile": "profiles/rs_step_kernel_c2_full.md"},
 }
@@ -490,7 +494,8 @@ def main():
     t = NCU_TRAFFIC["chain_fused_kernel"]
     roofline = roofline_entry(
         "chain_fused_kernel", chain_fused_bytes(N, count), ms_step, peak, peak_src,
-        t["bytes_per_element"] * count * N, f"ncu, {t['profile']}, scaled by elements",
+        t["captured"].get(w.name, t["bytes_per_element"] * count * N),
+        f"ncu, {t['profile']}" + (", this workload, inside the kernel" if w.name in t["captured"] else ", scaled by elements"),
         "4*count*nranks: every bf16 input read once, every bf16 output written once; hop messages stay in registers")
     roofline["ring_schedule_bytes_per_launch"] = ring_schedule_bytes(N, count, block)
     roofline["note"] = ("frac counts only bytes this kernel moves through HBM; against the ring schedule's "
