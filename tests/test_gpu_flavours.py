@@ -151,3 +151,39 @@ def test_fp8_flavour_bits_are_validated(gu):
     assert eq.allreduce_sim_flavour_workspace_bytes(4, 4 * 64, 64, 6 | eq.FLAVOUR_E4M3 | eq.FLAVOUR_E5M2) == 0
     assert eq.allreduce_sim_flavour_workspace_bytes(4, 4 * 64, 64, 6 | eq.FLAVOUR_E5M2) == binding.PIPELINE_MIN_WORKSPACE_BYTES
     assert eq.allreduce_sim_flavour_workspace_bytes(4, 4 * 64, 64, 32) == 0
+
+
+@pytest.mark.parametrize("flavour", (0, 5, 7, 6 | eq.FLAVOUR_E4M3))
+def test_flavours_in_place(gu, flavour):
+    """out[r] == in[r]: a tile's inputs are all read before any of its outputs is written."""
+    n, block = 8, 128
+    count = n * block * 21
+    x = wl.make_inputs(wl.Workload("t", n, count, block, "normal", seed=90 + flavour))
+    semi, qr, qa = decode(flavour)
+    exp = oracle.allreduce_variant(wl.as_u16(x), block, semi, qr, qa, payload=payload_of(flavour))["out"]
+    bufs = [gu.Guarded(2 * count) for _ in range(n)]
+    for r in range(n):
+        bufs[r].view(torch.bfloat16).copy_(x[r])
+    wb = eq.allreduce_sim_flavour_workspace_bytes(n, count, block, flavour, False)
+    ws = gu.Guarded(wb)
+    eq.allreduce_sim_flavour(bufs, bufs, n, count, block, flavour, ws, wb, False, gu.stream_handle())
+    torch.cuda.synchronize()
+    ws.check()
+    for b in bufs:
+        b.check()
+    gu.assert_same_words(torch.stack([b.view(torch.bfloat16) for b in bufs]), exp, f"flavour {flavour} in place")
+
+
+def test_host_entry_with_sixty_four_ranks(gu):
+    n, block = 64, 64
+    count = n * block * 3
+    x = wl.make_inputs(wl.Workload("t", n, count, block, "uniform", seed=17))
+    exp = oracle.allreduce(wl.as_u16(x), block)["out"]
+    h = x.clone().pin_memory()
+    sb = eq.allreduce_sim_host_staging_bytes(n, count)
+    stage = gu.Guarded(sb)
+    eq.allreduce_sim_host([h[r] for r in range(n)], [h[r] for r in range(n)], n, count, block, stage, sb,
+                          gu.stream_handle())
+    torch.cuda.synchronize()
+    stage.check()
+    gu.assert_same_words(h, exp, "host entry, 64 ranks, in place")
