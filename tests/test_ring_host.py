@@ -193,3 +193,73 @@ def test_peer_ring_setup_between_two_gloo_processes():
         assert calls[1]["timeout_ns"] == 5_000_000 and calls[0]["mailboxes"] == boxes
         assert log[-2:] == [("close", mapped), ("free", own)]              # unmap peers, then free the own one
         assert failed == ((1, 1, 0) if rank == 1 else None)               # only the rank whose wait ran out raises
+
+
+def _protocol_worker(rank, world, port, q, block, bps):
+    """One rank of the ring as a CPU process: the schedule and slot maps of RingLayout drive real
+    sends and receives (gloo); the arithmetic of every step is the oracle's per-step functions."""
+    import torch
+    import oracle
+    from paper_2506_17615_b200 import workloads as wl
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    count = world * bps * block
+    lay = RingLayout(world, count, block)
+    x = wl.as_u16(wl.make_rank(wl.Workload("t", world, count, block, "normal", seed=77), rank))
+    shard = lay.shard
+    slots = {}                                           # the mailbox: slot -> (codes, scales)
+
+    def exchange(dst, src, codes, scales):
+        """send one message to dst while receiving one from src (deadlock-free pairing)"""
+        out_c, out_s = torch.from_numpy(codes.copy()), torch.from_numpy(scales.copy())
+        in_c, in_s = torch.empty_like(out_c), torch.empty_like(out_s)
+        reqs = [dist.isend(out_c, dst), dist.isend(out_s, dst), dist.irecv(in_c, src), dist.irecv(in_s, src)]
+        for r_ in reqs:
+            r_.wait()
+        return in_c.numpy(), in_s.numpy()
+
+    for s in range(world):
+        k = lay.shard_sent(rank, s)
+        mine = x[k * shard:(k + 1) * shard]
+        if s == 0:
+            codes, scales = oracle.quantize_blocks(mine, block)
+        else:
+            c_in, s_in = slots[lay.recv_slot(s)]
+            codes, scales = oracle.rs_step(c_in, s_in, mine, block)
+        if s + 1 < world:
+            slots[lay.recv_slot(s + 1)] = exchange(lay.right(rank), lay.left(rank), codes, scales)
+        else:
+            assert k == rank                             # the reduced shard is the rank's own
+            slots[lay.gather_slot(k)] = (codes, scales)
+    # all-gather: every rank gets every reduced shard's message
+    for step in range(1, world):
+        dst, src = (rank + step) % world, (rank - step) % world
+        slots[lay.gather_slot(src)] = exchange(dst, src, *slots[lay.gather_slot(rank)])
+    out = np.concatenate([oracle.ag_dequant(*slots[lay.gather_slot(k)], block) for k in range(world)])
+    q.put((rank, out))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world", (2, 3))
+def test_ring_schedule_among_cpu_processes_equals_the_oracle_allreduce(world):
+    """The send/receive maps and mailbox slots, exercised by real message passing between processes,
+    reproduce the single-process oracle's AllReduce bit for bit on every rank."""
+    import oracle
+    from paper_2506_17615_b200 import workloads as wl
+    block, bps = 64, 3
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 33000 + os.getpid() % 2000 + world
+    procs = [ctx.Process(target=_protocol_worker, args=(r, world, port, q, block, bps)) for r in range(world)]
+    for p in procs:
+        p.start()
+    got = dict(q.get(timeout=240) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    x = wl.as_u16(wl.make_inputs(wl.Workload("t", world, world * bps * block, block, "normal", seed=77)))
+    exp = oracle.allreduce(x, block)["out"]
+    for r in range(world):
+        assert np.array_equal(got[r], exp[r]), f"rank {r}"
