@@ -185,3 +185,52 @@ def test_bench_ring_mode_with_a_single_rank():
     line = json.loads(out.stdout.strip().splitlines()[-1])
     assert line["failure"] is None and line["value"] > 0 and line["config"]["nranks"] == 1
     assert "ranks_here=1" in line["schedule"]
+
+
+def _mailbox_owner(nboxes, nbytes, handles_q, done_evt):
+    """A second process that owns mailboxes: allocates them, hands out their IPC handles, frees them at the end."""
+    mem = CudaIpcMemory()
+    ptrs = [mem.alloc_zeroed(nbytes) for _ in range(nboxes)]
+    handles_q.put([mem.export(p) for p in ptrs])
+    done_evt.wait(timeout=300)
+    for p in ptrs:
+        mem.free(p)
+
+
+def test_ring_through_mailboxes_owned_by_another_process(gu):
+    """Half of the mailboxes live in allocations of ANOTHER process, mapped here through CUDA IPC, as a peer
+    GPU's mailbox would be.  All ranks still run in one cooperative launch of this process (no kernel waits
+    on another launch); records, flags and acquire loads go through the IPC mappings."""
+    n, block = 4, 256
+    count = n * block * 9
+    lay = RingLayout(n, count, block)
+    ctx = mp.get_context("spawn")
+    handles_q, done = ctx.Queue(), ctx.Event()
+    owner = ctx.Process(target=_mailbox_owner, args=(2, lay.mailbox_bytes, handles_q, done))
+    owner.start()
+    mem = CudaIpcMemory()
+    mapped = []
+    try:
+        handles = handles_q.get(timeout=180)
+        mapped = [mem.open(h) for h in handles]
+        local = [torch.zeros(lay.mailbox_bytes, dtype=torch.uint8, device="cuda") for _ in range(2)]
+        boxes = [mapped[0], local[0], mapped[1], local[1]]           # ranks 0 and 2 receive in the other process's memory
+        x = wl.make_inputs(wl.Workload("t", n, count, block, "normal", seed=55))
+        xd = x.cuda()
+        outs = [gu.Guarded(2 * count) for _ in range(n)]
+        status = torch.zeros(4, dtype=torch.int32, device="cuda")
+        for epoch in (1, 2):
+            eq.ring_allreduce([xd[r] for r in range(n)], outs, 0, n, n, count, block, boxes, epoch, 0, status,
+                              gu.stream_handle())
+            torch.cuda.synchronize()
+            assert status.cpu().tolist()[0] == 0
+        exp = oracle.allreduce(wl.as_u16(x), block)["out"]
+        for o in outs:
+            o.check()
+        gu.assert_same_words(torch.stack([o.view(torch.bfloat16) for o in outs]), exp, "ring over IPC-mapped mailboxes")
+    finally:
+        for p in mapped:
+            mem.close(p)
+        done.set()
+        owner.join(timeout=60)
+    assert owner.exitcode == 0
