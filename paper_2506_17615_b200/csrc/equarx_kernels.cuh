@@ -5,8 +5,15 @@
 // Thread mapping, shared by every kernel: one lane owns 16 contiguous
 // elements (one 256-bit bf16 access, one 128-bit int8 access), so a block of
 // B elements is B/16 neighbouring lanes of one warp and the per-block max is
-// an in-lane max followed by log2(B/16) shuffles.  grid.y is the simulated
-// rank (or, in the all-gather, the shard); grid.x tiles the shard.
+// an in-lane max followed by log2(B/16) shuffles.
+//
+// Kernel families, all bit-identical in their results:
+//   rs_step_kernel, ag_dequant_kernel   one launch per ring step over all simulated ranks
+//                                       (grid.y = rank or shard, grid.x tiles the shard)
+//   pipelined_kernel, flavour_kernel    one persistent launch, every message written as a record
+//   chain_fused_kernel, flavour_fused_kernel   one persistent launch, messages kept in registers
+//   ring_rank_kernel                    one rank per device: peer mailboxes, per-tile flags
+//   bf16_step_kernel, bf16_gather_kernel        the unquantized comparator
 //
 // Every floating-point step that decides a bit of the result uses an explicit
 // round-to-nearest intrinsic, so the compiler cannot contract or reorder it:
@@ -21,10 +28,7 @@
 
 namespace equarx {
 
-#ifndef EQX_STEP_THREADS
-#define EQX_STEP_THREADS 256
-#endif
-constexpr int kThreads = EQX_STEP_THREADS;        // threads per CTA of the per-step kernels
+constexpr int kThreads = 256;        // threads per CTA of the per-step kernels (64/128/512 measured: not better)
 constexpr int kLaneElems = 16;       // elements per lane
 constexpr int kMaxRanks = 64;
 
@@ -1139,14 +1143,8 @@ __global__ void __launch_bounds__(kPipeThreads) flavour_fused_kernel(const __gri
 // A launch can host several consecutive ranks (ranks_here > 1): their CTAs are co-resident (the
 // launch is cooperative) and exchange through the same mailboxes, which is how the whole ring runs
 // and is checked on a single GPU.
-#ifndef EQX_RING_THREADS
-#define EQX_RING_THREADS 128
-#endif
-#ifndef EQX_RING_BATCH
-#define EQX_RING_BATCH 8
-#endif
-constexpr int kRingThreads = EQX_RING_THREADS;
-constexpr uint32_t kRingBatch = EQX_RING_BATCH;      // tiles whose records share one system-scope fence
+constexpr int kRingThreads = 128;       // 64 and 256 measured on one GPU: 5-8 % slower
+constexpr uint32_t kRingBatch = 8;      // tiles whose records share one system-scope fence (2 / 4 / 8: 920 / 731 / 686 us at 88 MB per rank)
 
 struct RingArgs {
     const void* in[kMaxRanks];       // input tensor of hosted rank rank_first + i
