@@ -29,6 +29,7 @@ _BINDING_NAMES = (
     "allreduce_sim_host",
     "allreduce_sim_host_staging_bytes",
     "allreduce_sim_pipelined",
+    "allreduce_sim_pipelined_unordered",
     "allreduce_sim_pipelined_workspace_bytes",
     "allreduce_sim_range",
     "allreduce_sim_static",

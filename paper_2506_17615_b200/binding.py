@@ -27,6 +27,7 @@ EXPORTS = (
     "equarx_allreduce_sim_pipelined",
     "equarx_allreduce_sim_pipelined_workspace_bytes",
     "equarx_allreduce_sim_host",
+    "equarx_allreduce_sim_pipelined_unordered",
     "equarx_ring_allreduce",
     "equarx_ring_mailbox_bytes",
     "equarx_allreduce_sim_host_staging_bytes",
@@ -59,6 +60,7 @@ def _load():
     lib.equarx_allreduce_sim_pipelined.argtypes = [vp, vp, ci, sz, ci, vp, sz, ci, vp]
     lib.equarx_allreduce_sim_pipelined_workspace_bytes.argtypes = [ci, sz, ci, ci]
     lib.equarx_allreduce_sim_pipelined_workspace_bytes.restype = sz
+    lib.equarx_allreduce_sim_pipelined_unordered.argtypes = [vp, vp, ci, sz, ci, vp]
     lib.equarx_allreduce_sim_host.argtypes = [vp, vp, ci, sz, ci, vp, sz, vp]
     lib.equarx_allreduce_sim_host_staging_bytes.argtypes = [ci, sz]
     lib.equarx_allreduce_sim_host_staging_bytes.restype = sz
@@ -147,6 +149,14 @@ def allreduce_sim_pipelined(in_bf16, out_bf16, nranks, count, block, workspace, 
     _check(lib.equarx_allreduce_sim_pipelined(_table(in_bf16), _table(out_bf16), nranks, count, block,
                                               _ptr(workspace), workspace_bytes, int(bool(keep_trace)), _ptr(stream)),
            "equarx_allreduce_sim_pipelined")
+
+
+def allreduce_sim_pipelined_unordered(in_bf16, out_bf16, nranks, count, block, stream=0):
+    """The chain-fused single launch for a call that is independent of the stream's unfinished earlier
+    work (the caller's promise): starts while that work is finishing, completes after it."""
+    _check(lib.equarx_allreduce_sim_pipelined_unordered(_table(in_bf16), _table(out_bf16), nranks, count, block,
+                                                        _ptr(stream)),
+           "equarx_allreduce_sim_pipelined_unordered")
 
 
 def allreduce_sim_host_staging_bytes(nranks, count):

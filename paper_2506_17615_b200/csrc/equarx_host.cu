@@ -414,7 +414,8 @@ size_t equarx_allreduce_sim_pipelined_workspace_bytes(int nranks, size_t count, 
 namespace {
 // the single-launch schedule on validated arguments (workspace: the trace, or unused)
 int launch_pipelined(const void* const* in_bf16, void* const* out_bf16, int nranks, size_t count, int block,
-                     void* workspace, int keep_trace, cudaStream_t stream, bool quantized = true) {
+                     void* workspace, int keep_trace, cudaStream_t stream, bool quantized = true,
+                     bool unordered = false) {
     const uint32_t N = uint32_t(nranks);
     const size_t shard = count / N;
     PipeArgs a = {};
@@ -424,6 +425,7 @@ int launch_pipelined(const void* const* in_bf16, void* const* out_bf16, int nran
         a.out[r] = out_bf16[r];
     }
     a.records = static_cast<char*>(workspace);
+    a.unordered = (unordered && !keep_trace) ? 1u : 0u;
     a.shard = shard;
     a.tiles_per_shard = (shard + kTileElems - 1) / kTileElems;
     a.nranks = N;
@@ -490,6 +492,13 @@ int equarx_allreduce_sim_pipelined(const void* const* in_bf16, void* const* out_
     if (!aligned(workspace, 32)) return EQUARX_ERR_ALIGN;
     if (int st = check_tables(in_bf16, out_bf16, nranks, 2 * count, workspace, need)) return st;
     return launch_pipelined(in_bf16, out_bf16, nranks, count, block, workspace, keep_trace, stream);
+}
+
+int equarx_allreduce_sim_pipelined_unordered(const void* const* in_bf16, void* const* out_bf16, int nranks,
+                                             size_t count, int block, equarx_stream_t stream) {
+    if (int st = check_sim_shape(nranks, count, block)) return st;
+    if (int st = check_tables(in_bf16, out_bf16, nranks, 2 * count, nullptr, 0)) return st;
+    return launch_pipelined(in_bf16, out_bf16, nranks, count, block, nullptr, 0, stream, true, true);
 }
 
 size_t equarx_allreduce_sim_host_staging_bytes(int nranks, size_t count) {

@@ -482,6 +482,7 @@ struct PipeArgs {
     uint64_t shard;
     uint64_t tiles_per_shard;        // 512-element tiles per shard (the last one may be ragged)
     uint32_t nranks;
+    uint32_t unordered;              // chain-fused form only: do not wait for the stream's earlier work before starting
     float neg_zero;                  // -0.0f, opaque to the compiler (see quantize_lane)
 };
 
@@ -731,8 +732,13 @@ __global__ void __launch_bounds__(kPipeThreads, MINB) chain_fused_kernel(const _
     const uint64_t groups = a.shard >> 4;
     const uint64_t tiles = a.tiles_per_shard * N;
 
+    // Ordered (the default): nothing is read before the previous kernel of the stream has completed.
+    // Unordered: the caller vouches that no unfinished earlier work of the stream writes the inputs or
+    // touches the outputs, so the grid starts while that work is still finishing (this removes the
+    // idle gap between back-to-back independent AllReduces) and waits for it only before it exits, so
+    // that whatever follows in the stream still sees all earlier work complete.
     pdl_launch_dependents();
-    pdl_wait_prior_grid();           // nothing is read before the previous kernel of the stream has completed
+    if (!a.unordered) pdl_wait_prior_grid();
 
     // byte offset of this lane's group of a tile in every rank's tensor; ~0 past the end of a ragged last tile
     auto offset_of = [&](uint64_t tile_, uint32_t& k_) -> uint64_t {
@@ -808,6 +814,7 @@ __global__ void __launch_bounds__(kPipeThreads, MINB) chain_fused_kernel(const _
         if (off != ~uint64_t(0))
             for (uint32_t r = 0; r < N; ++r) st_stream_256(static_cast<char*>(a.out[r]) + off, o);
     }
+    if (a.unordered) pdl_wait_prior_grid();
 }
 
 // ---------------------------------------------------------------- the other flavours

@@ -479,6 +479,42 @@ def test_runs_on_the_stream_it_is_given(gu):
     gu.assert_same_words(out, exp, "side stream")
 
 
+def test_unordered_single_launch_back_to_back_on_independent_tensors(gu):
+    """equarx_allreduce_sim_pipelined_unordered: thirty calls back to back on six independent tensor sets
+    (each launch may start while its predecessors are still finishing) give the oracle's bits, and work
+    enqueued afterwards still finds ALL earlier work complete: a large ordered AllReduce, a small unordered
+    one that finishes its own work first, then a copy of the large one's output."""
+    n, block = 8, 256
+    count = n * block * 64
+    xs = [wl.make_inputs(wl.Workload("t", n, count, block, "normal", seed=300 + i)) for i in range(6)]
+    exp = [oracle.allreduce(wl.as_u16(x), block)["out"] for x in xs]
+    xd = [x.cuda() for x in xs]
+    outs = [torch.zeros_like(x) for x in xd]
+    s = gu.stream_handle()
+    for i in range(30):
+        j = i % 6
+        eq.allreduce_sim_pipelined_unordered([xd[j][r] for r in range(n)], [outs[j][r] for r in range(n)], n, count,
+                                             block, s)
+    torch.cuda.synchronize()
+    for j in range(6):
+        gu.assert_same_words(outs[j], exp[j], f"unordered, set {j}")
+
+    big = wl.make_inputs(wl.C2, device="cuda")                 # 8 x 15.7 MB: tens of microseconds
+    big_out = torch.zeros_like(big)
+    wb = eq.allreduce_sim_pipelined_workspace_bytes(8, wl.C2.count, 256, False)
+    ws = torch.empty(wb, dtype=torch.uint8, device="cuda")
+    small_out = torch.zeros_like(xd[0])
+    torch.cuda.synchronize()
+    eq.allreduce_sim_pipelined([big[r] for r in range(8)], [big_out[r] for r in range(8)], 8, wl.C2.count, 256, ws, wb,
+                               False, s)
+    eq.allreduce_sim_pipelined_unordered([xd[0][r] for r in range(n)], [small_out[r] for r in range(n)], n, count, block, s)
+    snapshot = big_out.clone()                                 # ordinary stream work after the unordered call
+    torch.cuda.synchronize()
+    assert torch.equal(snapshot.view(torch.int16), big_out.view(torch.int16))
+    gu.assert_same_words(snapshot, oracle.allreduce(wl.as_u16(big), 256)["out"], "work after an unordered call")
+    gu.assert_same_words(small_out, exp[0], "the unordered call itself")
+
+
 def test_schedules_can_be_recorded_in_a_cuda_graph(gu):
     """The simulation calls only enqueue launches on the given stream (no synchronisation, no allocation),
     so stream capture records them; replaying the graph on new data gives the oracle's bits.  Small
