@@ -110,6 +110,43 @@ int main(void)
             return 1;
         CHECK_CUDA(cudaFree(stage));
     }
+    /* the unordered single launch and the ring with one rank per device (all ranks hosted by this process) */
+    {
+        CHECK_EQ(equarx_oracle_allreduce((const uint16_t *const *)h_in, h_ref, N, count, BLOCK, NULL, NULL, NULL));
+        for (int r = 0; r < N; ++r) CHECK_CUDA(cudaMemset(d_out[r], 0, count * 2));
+        CHECK_EQ(equarx_allreduce_sim_pipelined_unordered((const void *const *)d_in, d_out, N, count, BLOCK, NULL));
+        CHECK_CUDA(cudaDeviceSynchronize());
+        for (int r = 0; r < N; ++r) {
+            CHECK_CUDA(cudaMemcpy(h_out[r], d_out[r], count * 2, cudaMemcpyDeviceToHost));
+            if (memcmp(h_out[r], h_ref[r], count * 2) != 0) { fprintf(stderr, "unordered launch: rank %d differs\n", r); return 1; }
+        }
+        void *boxes[N];
+        uint32_t *status, h_status[4];
+        const size_t box_bytes = equarx_ring_mailbox_bytes(N, count, BLOCK);
+        if (box_bytes == 0) return 1;
+        for (int r = 0; r < N; ++r) {
+            CHECK_CUDA(cudaMalloc(&boxes[r], box_bytes));
+            CHECK_CUDA(cudaMemset(boxes[r], 0, box_bytes));
+            CHECK_CUDA(cudaMemset(d_out[r], 0, count * 2));
+        }
+        CHECK_CUDA(cudaMalloc((void **)&status, 16));
+        CHECK_CUDA(cudaMemset(status, 0, 16));
+        for (uint32_t epoch = 1; epoch <= 2; ++epoch)
+            CHECK_EQ(equarx_ring_allreduce((const void *const *)d_in, d_out, 0, N, N, count, BLOCK, boxes, epoch, 0, status,
+                                           NULL));
+        CHECK_CUDA(cudaDeviceSynchronize());
+        CHECK_CUDA(cudaMemcpy(h_status, status, 16, cudaMemcpyDeviceToHost));
+        if (h_status[0] != 0) { fprintf(stderr, "ring: status %u\n", h_status[0]); return 1; }
+        for (int r = 0; r < N; ++r) {
+            CHECK_CUDA(cudaMemcpy(h_out[r], d_out[r], count * 2, cudaMemcpyDeviceToHost));
+            if (memcmp(h_out[r], h_ref[r], count * 2) != 0) { fprintf(stderr, "ring: rank %d differs\n", r); return 1; }
+            CHECK_CUDA(cudaFree(boxes[r]));
+        }
+        if (equarx_ring_allreduce((const void *const *)d_in, d_out, 0, N, N, count, BLOCK, boxes, 0, 0, status, NULL)
+            != EQUARX_ERR_COUNT)           /* epoch 0 is refused */
+            return 1;
+        CHECK_CUDA(cudaFree(status));
+    }
     /* an error path: a count that is not a multiple of nranks * block is refused before any launch */
     if (equarx_allreduce_sim((const void *const *)d_in, d_out, N, count + BLOCK, BLOCK, d_out[0], 1 << 20, 0, NULL)
         != EQUARX_ERR_COUNT)
