@@ -709,7 +709,7 @@ __global__ void __launch_bounds__(kPipeThreads, EQX_PIPE_MINBLOCKS) pipelined_ke
 // for the sending rank can go on, as the receiving rank, with the fused multiply-add on that
 // rank's counterpart: the hop message of a group (its codes, as the fp32 values of the int8
 // codes, and the block's scale) stays in that lane's registers and is never stored.  Codes,
-// scales and outputs are bit for bit those of pipelined_kernel<LPB, true>, which writes every
+// scales and outputs are bit for bit those of pipelined_kernel<LPB>, which writes every
 // message as a record and is the witness of that; what this kernel moves through HBM is the
 // bf16 inputs once and the bf16 outputs once (4 bytes per element of every rank).
 // The bf16 shard of the next rank of the chain is in flight while a step computes; DEPTH is the
