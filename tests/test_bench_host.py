@@ -111,3 +111,17 @@ def test_bench_line_on_the_gpu_is_consistent():
     assert line["parity"]["verdict"] == "bit-exact" and line["parity"]["checked_words"] == n * count
     assert line["e2e"]["h2d_bytes_per_step"] == 2 * count * n == line["e2e"]["d2h_bytes_per_step"]
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] == 1
+
+
+@pytest.mark.gpu
+def test_sweep_point_runs_and_accounts_bytes_per_schedule():
+    """One small point of the message-size sweep: three schedules timed, each fraction against its own bytes."""
+    from paper_2506_17615_b200 import sweep
+    rec = sweep.run_point(4, 1 << 20, 256, "uniform", 6534.1)
+    n = (1 << 20) // 2
+    for key, nbytes in (("pipelined", 4 * n * 4), ("by_steps", n * 4 * (6 + 8 / 256)), ("bf16_sim", n * (8 * 4 - 4))):
+        leg = rec[key]
+        assert leg["ms"] > 0
+        assert leg["frac"] == pytest.approx(nbytes / (leg["ms"] * 1e-3) / 1e9 / 6534.1, rel=1e-9)
+        assert leg["gbs_in"] == pytest.approx(2 * n * 4 / (leg["ms"] * 1e-3) / 1e9, rel=1e-9)
+    assert sweep.run_point(3, 1 << 20, 256, "uniform", 6534.1) is None       # not divisible by nranks * block
